@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the AdLoCo hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input:
+  1. norm test on materialised per-sample gradients (B=64, P=2^24 fp32), with the
+     batch decision for eta in {0.1, 0.5, 1.0} from one pass over the gradients;
+  2. outer step over K=8 bf16 instances of a 124M-parameter vector (fp32 global
+     parameters and momentum, lr 0.7, Nesterov momentum 0.9), in place;
+  3. Gram-identity per-sample norms + mean-gradient GEMM for one linear layer
+     (X bf16 [32,1024,768], Delta bf16 [32,1024,3072]), accumulated into a
+     switch-mode accumulator and finalised into one test.
+The headline value is the HBM throughput of the streaming part (1 + 2):
+algorithmic bytes / device time.  The tensor-core part is reported beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (under torchrun) every rank runs the same workload on its own GPU
+(the path has no exchange step: weak scaling, no collective on the data path);
+the time is the max over ranks and the value the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2508_18182_b200 import workloads as W  # noqa: E402
+
+METRIC = "norm-test + outer-merge HBM GB/s"
+UNIT = "GB/s"
+
+# the streaming workload the metric is quoted on
+NT_B, NT_P = 64, 1 << 24
+OUT_K, OUT_P = 8, W.GPT2_SMALL_P
+ETAS = (0.1, 0.5, 1.0)
+LR, MU = 0.7, 0.9
+# the tensor-core workload
+GR_B, GR_T, GR_DIN, GR_DOUT = 32, 1024, 768, 3072
+
+
+def algorithmic_bytes():
+    nt = 4 * NT_B * NT_P                               # every gradient element read once
+    outer = (2 * OUT_K + 8) * OUT_P + 8 * OUT_P        # K bf16 instances + theta + v read; theta + v written
+    return nt, outer
+
+
+def gram_flops():
+    sym = GR_B * GR_T * (GR_T + 1) * (GR_DIN + GR_DOUT)          # symmetric half of both Gram products
+    tiles = (GR_T // 128) * (GR_T // 128 + 1) // 2
+    executed = 2 * GR_B * tiles * 128 * 128 * (GR_DIN + GR_DOUT)  # at 128-token tile granularity
+    mean_grad = 2 * GR_B * GR_T * GR_DIN * GR_DOUT
+    return sym, executed, mean_grad
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------
+# clocks during the timed region
+# ------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------
+# reference arm / CPU baseline: the fp64 oracle on the host cores
+# ------------------------------------------------------------------------------------
+def oracle_sample_run(steps: int, warmup: int):
+    """Times the oracle, as it stands, on a bounded sample of the streaming
+    workload: the norm test on B=64 x P=2^19 and the outer step on K=8 x P=2^21.
+    Returns (GB/s over the sample's algorithmic bytes, ms per step, threads)."""
+    import numpy as np
+    import oracle.adloco_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = 1
+    sP, oP = 1 << 19, 1 << 21
+    G = W.to_numpy(W.per_sample_grads(NT_B, sP, sigma=0.5, seed=1))
+    theta, inst, mom = W.outer_state(OUT_K, oP, inst_dtype=torch.bfloat16, seed=2)
+    th, v, ins = W.to_numpy(theta), W.to_numpy(mom), [W.to_numpy(t) for t in inst]
+    nbytes = 4 * NT_B * sP + (2 * OUT_K + 8) * oP + 8 * oP
+
+    def one():
+        r = O.norm_test(G, eta=ETAS[0], b_cur=NT_B, b_max=32)
+        for eta in ETAS[1:]:
+            O.decide(r.sum_sqnorm, r.mean_sqnorm, r.variance, NT_B, eta=eta, b_cur=NT_B, b_max=32)
+        O.outer_step(th, ins, v, lr=LR, momentum=MU, nesterov=True)
+
+    for _ in range(warmup):
+        one()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    sample = f"norm test B={NT_B} P=2^19 fp32 + outer step K={OUT_K} bf16 P=2^21 (1/32 resp. 1/59 of the workload)"
+    return nbytes / dt / 1e9, dt * 1e3, threads, sample
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 5))
+    warm = max(1, min(args.warmup, 2))
+    gbs, ms, threads, sample = oracle_sample_run(steps, warm)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": workload_config(),
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config():
+    return {"workload": "configs[1] streaming scale-up: norm test B=64 P=16,777,216 fp32 (eta 0.1/0.5/1.0) + "
+                        "outer step K=8 bf16 P=124,439,808 (fp32 theta and momentum, lr 0.7, Nesterov 0.9); "
+                        "plus configs[2] Gram layer B=32 T=1024 768->3072 bf16 for the tensor-core figure",
+            "l2": "inputs larger than L2 (4.3 GB + 4.0 GB + 0.25 GB per step), no flush needed",
+            "parallelism": "replicas (no exchange step on the path)"}
+
+
+# ------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------
+def run_ours(args, rank, world, local_rank):
+    from paper_2508_18182_b200 import binding as A
+    from paper_2508_18182_b200.build import build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    ctx = A.Context(local_rank)
+
+    # ---- resident inputs
+    G = W.per_sample_grads(NT_B, NT_P, sigma=0.5, seed=10 + rank, device=dev)
+    theta, inst, mom = W.outer_state(OUT_K, OUT_P, inst_dtype=torch.bfloat16, seed=20 + rank, device=dev)
+    X, D = W.linear_layer(GR_B, GR_T, GR_DIN, GR_DOUT, seed=30 + rank, device=dev)
+    S_layer = torch.zeros(GR_DOUT, GR_DIN, device=dev)
+    n_layer = torch.zeros(GR_B, device=dev)
+    acc = A.Accumulator(ctx, [S_layer])
+    params = [A.make_params(eta, b_cur=NT_B, b_max=32) for eta in ETAS]
+    gparams = A.make_params(0.5, b_cur=GR_B, b_max=32)
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(marks=None):
+        if marks is not None:
+            marks["nt0"].record(stream)
+        ctx.norm_test(G, params[0], sync=False)
+        if marks is not None:
+            marks["nt1"].record(stream)
+        for p in params[1:]:
+            ctx.test_decide(p, sync=False)
+        if marks is not None:
+            marks["os0"].record(stream)
+        ctx.outer_step(inst, theta, mom, lr=LR, momentum=MU, nesterov=True)
+        if marks is not None:
+            marks["os1"].record(stream)
+        acc.reset()
+        ctx.gram_sqnorm(X, D, n_layer, grad_sum=S_layer, accumulate_sum=True)
+        acc.accumulate(per_sample_sqnorm=n_layer)
+        acc.finalize(gparams, sync=False)
+        if marks is not None:
+            marks["gr1"].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    marks = [{k: ev() for k in ("nt0", "nt1", "os0", "os1", "gr1")} for _ in range(args.steps)]
+    launches0 = ctx.launch_count
+    torch.cuda.synchronize()
+    t_begin, t_end = ev(), ev()
+    t_begin.record(stream)
+    for s in range(args.steps):
+        step(marks[s])
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    if use_dist:
+        import torch.distributed as dist
+        dist.barrier()
+    clocks = sampler.stop()
+    launches = ctx.launch_count - launches0
+    last = ctx._read_result()
+
+    total_ms = t_begin.elapsed_time(t_end)
+    nt_ms = sum(m["nt0"].elapsed_time(m["nt1"]) for m in marks) / args.steps
+    os_ms = sum(m["os0"].elapsed_time(m["os1"]) for m in marks) / args.steps
+    stream_ms = sum(m["nt0"].elapsed_time(m["os1"]) for m in marks) / args.steps
+    gram_ms = sum(m["os1"].elapsed_time(m["gr1"]) for m in marks) / args.steps
+    times = torch.tensor([total_ms, stream_ms, gram_ms, nt_ms, os_ms], dtype=torch.float64, device=dev)
+    if use_dist:
+        import torch.distributed as dist
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, stream_ms, gram_ms, nt_ms, os_ms = times.tolist()
+
+    nt_bytes, os_bytes = algorithmic_bytes()
+    peaks = load_peaks()
+    value = world * (nt_bytes + os_bytes) / (stream_ms * 1e-3) / 1e9
+    sym, executed, mg = gram_flops()
+
+    # ---- end to end through the host-memory entry points (rank-local pinned buffers)
+    e2e = None
+    if not args.no_e2e:
+        Gh = torch.empty((NT_B, NT_P), dtype=torch.float32).pin_memory()
+        Gh.copy_(G)
+        th_h = theta.cpu().pin_memory()
+        v_h = mom.cpu().pin_memory()
+        inst_h = [t.cpu().pin_memory() for t in inst]
+        reps = max(1, min(args.steps, 3))
+        ctx.norm_test_host(Gh, params[0])                   # warm-up: allocates the staging buffers
+        ctx.outer_step_host(inst_h, th_h, v_h, lr=LR, momentum=MU)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            ctx.norm_test_host(Gh, params[0])
+            for p in params[1:]:
+                pass                                        # the eta sweep needs no further data movement
+            ctx.outer_step_host(inst_h, th_h, v_h, lr=LR, momentum=MU)
+        torch.cuda.synchronize()
+        e2e_s = torch.tensor([(time.perf_counter() - t0) / reps], dtype=torch.float64, device=dev)
+        if use_dist:
+            dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * (nt_bytes + os_bytes) / e2e_s.item() / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": nt_bytes + (2 * OUT_K + 8) * OUT_P,
+               "d2h_bytes_per_step": 8 * OUT_P + 80, "ms_per_step": e2e_s.item() * 1e3, "steps": reps}
+        del Gh, th_h, v_h, inst_h
+
+    if rank != 0:
+        return
+    nt_gbs = nt_bytes / (nt_ms * 1e-3) / 1e9
+    os_gbs = os_bytes / (os_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(),
+        "clocks": clocks,
+        "gpu_launches": launches,
+        "stream_ms_per_step": stream_ms,
+        "roofline": {"bound": "hbm", "kernel": "norm_test_kernel", "achieved": nt_gbs, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": nt_gbs / peaks["hbm_gbs"], "traffic": None,
+                     "peak_source": peaks["source"], "ms_per_launch": nt_ms, "algorithmic_bytes": nt_bytes},
+        "kernels": {
+            "outer_step_kernel": {"bound": "hbm", "achieved": os_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                  "frac": os_gbs / peaks["hbm_gbs"], "ms_per_launch": os_ms,
+                                  "algorithmic_bytes": os_bytes},
+            "gram_path": {"bound": "tensor", "ms_per_step": gram_ms,
+                          "achieved": (sym + mg) / (gram_ms * 1e-3) / 1e12,
+                          "executed_tflops": (executed + mg) / (gram_ms * 1e-3) / 1e12,
+                          "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                          "frac": (sym + mg) / (gram_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                          "algorithmic_flops": sym + mg, "includes": "gram + mean-grad + accumulate + finalize"},
+        },
+        "last_result": {"stat": last.stat, "b_req": last.b_req, "flags": last.flags},
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        gbs, ms, threads, sample = oracle_sample_run(2, 1)
+        line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

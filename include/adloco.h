@@ -1,0 +1,251 @@
+/*
+ * adloco.h -- C ABI of the AdLoCo hot path on one B200 (sm_100a).
+ *
+ * The library computes, with hand-written CUDA kernels,
+ *   - the approximate norm test that sizes the next local batch
+ *     (paper, Section "Norm test": sigma^2_B, the batch rule b_{k+1}),
+ *   - switch mode's accumulation of the test sums over micro-batches
+ *     (Section "Mode switching"; first branch of Algorithm 3),
+ *   - the outer step over K model instances (last loop of Algorithm 3),
+ *   - the trainer merge (Algorithms 1 and 2).
+ *
+ * Conventions for every entry point
+ *   - Returns an adloco_status (0 = ok, negative = error).  No exception, abort
+ *     or trap crosses this boundary.  Argument errors are found on the host
+ *     before anything is launched.
+ *   - "dev" pointers are device memory owned by the caller; "host" pointers are
+ *     host memory owned by the caller.  Base pointers of vector data must be
+ *     16-byte aligned unless an entry point says otherwise (ADLOCO_ERR_ALIGNMENT
+ *     if not).  The library owns only the workspace inside an adloco_ctx.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream) and is asynchronous unless stated.  One ctx must
+ *     not be used from two streams at the same time: its workspace is shared.
+ *   - Sizes are int64_t element counts; all byte offsets are 64-bit inside.
+ *   - There is no CPU fallback: without a usable CUDA device the calls fail
+ *     with ADLOCO_ERR_CUDA.
+ */
+#ifndef ADLOCO_H
+#define ADLOCO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct adloco_ctx adloco_ctx;     /* device id, workspace, cached tensor maps */
+typedef struct adloco_accum adloco_accum; /* switch-mode accumulator state */
+
+typedef enum {
+    ADLOCO_OK = 0,
+    ADLOCO_ERR_INVALID_ARG = -1,
+    ADLOCO_ERR_UNSUPPORTED = -2, /* a shape the kernels do not take; never a silent fallback */
+    ADLOCO_ERR_ALIGNMENT = -3,
+    ADLOCO_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed; see adloco_last_cuda_error */
+    ADLOCO_ERR_WORKSPACE = -5,
+    ADLOCO_ERR_TIMEOUT = -6      /* a bounded wait inside a kernel ran out (device status word) */
+} adloco_status;
+
+typedef enum { ADLOCO_F32 = 0, ADLOCO_BF16 = 1 } adloco_dtype;
+
+enum {
+    ADLOCO_FLAG_GROW = 1,       /* b_req > b_cur */
+    ADLOCO_FLAG_ACCUMULATE = 2, /* switch mode: b_req > switch_n * b_max */
+    ADLOCO_FLAG_UNDEFINED = 4,  /* batch_count - ddof <= 0: no variance; b_req = max(1, b_cur) */
+    ADLOCO_FLAG_ZERO_MEAN = 8   /* ||gbar||^2 == 0: stat = +inf, b_req = b_cap or INT64_MAX */
+};
+
+/* Parameters of the batch rule and of switch mode.
+ *   eta      threshold of the norm test, > 0 and finite
+ *   ddof     variance normaliser is (b - ddof); 1 = unbiased sample variance
+ *   b_cur    current batch size (only for the GROW flag and the UNDEFINED case)
+ *   b_max    largest micro-batch the hardware holds (max_batch), >= 1
+ *   b_cap    upper clamp on b_req, 0 = none
+ *   switch_n switch multiplier n (the paper uses 2), >= 1 */
+typedef struct {
+    double eta;
+    int32_t ddof;
+    int32_t switch_n;
+    int64_t b_cur;
+    int64_t b_max;
+    int64_t b_cap;
+} adloco_test_params;
+
+/* Sufficient statistics of one test (device memory, written by the kernels).
+ *   sum_sqnorm  Q   = sum_i ||g_i||^2
+ *   sum_sq_gsum      ||sum_i g_i||^2  (so ||gbar||^2 = sum_sq_gsum / b^2)
+ *   centred_ss       sum_i ||g_i - gbar||^2 computed column-centred; valid iff has_centred
+ *   batch_count b */
+typedef struct {
+    double sum_sqnorm;
+    double sum_sq_gsum;
+    double centred_ss;
+    int64_t batch_count;
+    int32_t has_centred;
+    int32_t device_status; /* 0, or an adloco_status raised on the device */
+} adloco_test_sums;
+
+/* Outcome of the test.  mean_sqnorm = ||gbar||^2, variance = sigma^2_B,
+ * stat = variance / (eta^2 mean_sqnorm), b_req = max(1, ceil(stat)) clamped by b_cap;
+ * accum_steps / b_micro are the switch-mode plan. */
+typedef struct {
+    double sum_sqnorm;
+    double mean_sqnorm;
+    double variance;
+    double stat;
+    int64_t batch_count;
+    int64_t b_req;
+    int64_t accum_steps;
+    int64_t b_micro;
+    uint32_t flags;
+    int32_t device_status;
+} adloco_test_result;
+
+/* ---- context ------------------------------------------------------------ */
+
+/* Creates a context on CUDA device `device` (allocates a few MB of workspace;
+ * synchronous).  *out is NULL on failure. */
+int adloco_create(adloco_ctx** out, int device);
+/* Frees the workspace.  The caller must have synchronised every stream that used it. */
+int adloco_destroy(adloco_ctx* ctx);
+const char* adloco_status_string(int status);
+/* Text of the last CUDA error seen by this ctx ("" if none); valid until the next call. */
+const char* adloco_last_cuda_error(const adloco_ctx* ctx);
+/* Number of kernel launches this ctx has enqueued so far. */
+int64_t adloco_launch_count(const adloco_ctx* ctx);
+
+/* ---- norm test on materialised per-sample gradients ---------------------- */
+
+/* Section "Norm test" (Eq. 1, sigma^2_B, b_{k+1}) followed by the switch-mode
+ * plan (Section "Mode switching").
+ *   grads              dev, [B, P] row-major, row i = g_i, row pitch `row_stride`
+ *                      elements (>= P), dtype F32 only.  128-bit loads are used when the
+ *                      base is 16-byte aligned and the pitch is a multiple of 4 (and
+ *                      grad_sum, if given, is 16-byte aligned); otherwise a slower
+ *                      32-bit path runs.  1 <= B <= 4096.
+ *   per_sample_sqnorm  dev [B] float, receives n_i = ||g_i||^2; may be NULL
+ *   grad_sum           dev [P] float, receives S = sum_i g_i; may be NULL
+ *   sums_dev           dev, receives the sufficient statistics; may be NULL
+ *   result_dev         dev, receives the decision; required
+ *   result_host        host (pinned for a truly asynchronous copy), filled by an async
+ *                      copy on `stream`, valid after the stream is synchronised; may be NULL
+ * One pass over G: per-row sum of squares, per-column sum and column-centred
+ * sum of squares, fp32 inside a thread, fp64 across threads and blocks (fixed
+ * order: results are run-to-run deterministic).  B >= 1, P >= 1. */
+int adloco_norm_test(adloco_ctx* ctx, const void* grads, adloco_dtype dtype, int64_t B, int64_t P,
+                     int64_t row_stride, const adloco_test_params* params, float* per_sample_sqnorm,
+                     float* grad_sum, adloco_test_sums* sums_dev, adloco_test_result* result_dev,
+                     adloco_test_result* result_host, void* stream);
+
+/* The batch rule and switch plan alone, from sufficient statistics already on
+ * the device (e.g. to sweep eta without re-reading the gradients). */
+int adloco_test_decide(adloco_ctx* ctx, const adloco_test_sums* sums_dev, const adloco_test_params* params,
+                       adloco_test_result* result_dev, adloco_test_result* result_host, void* stream);
+
+/* Same as adloco_norm_test with `grads_host` in HOST memory ([B, P], pitch
+ * row_stride): the library stages column panels through device buffers it owns,
+ * overlapping the copies with the reduction.  Synchronous: on return
+ * *result_host (required) and the optional host outputs per_sample_sqnorm_host
+ * [B] are valid. */
+int adloco_norm_test_host(adloco_ctx* ctx, const float* grads_host, int64_t B, int64_t P, int64_t row_stride,
+                          const adloco_test_params* params, float* per_sample_sqnorm_host,
+                          adloco_test_result* result_host, void* stream);
+
+/* ---- per-sample norms of a linear layer via the Gram identity ------------ */
+
+/* For a linear layer y = W x and a batch of B sequences of T tokens, sample i
+ * has weight gradient G_i = sum_t delta_{i,t} x_{i,t}^T (Eq. 1 applied to W).
+ * This call computes, on the tensor cores,
+ *   n_i = ||G_i||_F^2 = sum_{t,s} (x_t . x_s)(delta_t . delta_s)     (Gram identity)
+ *   S   = sum_i G_i = Delta^T X  ([d_out, d_in], fp32 accumulate)     (optional)
+ *   X  dev bf16 [B, T, d_in]  row-major (features contiguous)
+ *   D  dev bf16 [B, T, d_out] row-major
+ *   per_sample_sqnorm  dev [B] float; overwritten, or += when accumulate_norms != 0
+ *   grad_sum           dev [d_out, d_in] float, may be NULL; overwritten, or += when
+ *                      accumulate_sum != 0
+ * d_in and d_out must be multiples of 8 (ADLOCO_ERR_UNSUPPORTED otherwise); any
+ * B, T >= 1.  bf16 x bf16 products are exact in fp32; accumulation is fp32. */
+int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                       int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
+                       int accumulate_sum, void* stream);
+
+/* ---- switch-mode accumulation -------------------------------------------- */
+
+/* Accumulator of the test sums over the micro-batches of one large batch:
+ * Q = sum n_i, the batch count, and the gradient-sum buffers S (one per
+ * parameter buffer; caller-owned dev float arrays that the accumulator borrows).
+ * adloco_accum_create copies the n_bufs pointers/sizes (host arrays) and
+ * allocates a small device state; synchronous. */
+int adloco_accum_create(adloco_ctx* ctx, adloco_accum** out, float* const* sum_bufs, const int64_t* sum_sizes,
+                        int32_t n_bufs);
+/* Zeroes Q, the count and every S buffer (async on stream). */
+int adloco_accum_reset(adloco_ctx* ctx, adloco_accum* acc, void* stream);
+int adloco_accum_destroy(adloco_accum* acc);
+
+/* Adds one micro-batch (Algorithm 3's g <- g + grad L(x; B), applied to the
+ * test sums).  Two forms:
+ *  (a) grads != NULL: materialised micro-batch [b_micro, P] float (pitch row_stride),
+ *      P == sum_sizes[0] and n_bufs == 1.  One pass adds sum_i g_i into S, sum_i n_i
+ *      into Q, and keeps the centred sum of squares exact across micro-batches by
+ *      the pairwise update  css += css_mb + (c b/(c+b)) ||mean_mb - mean_so_far||^2.
+ *      per_sample_sqnorm (dev [b_micro], may be NULL) receives this micro-batch's n_i.
+ *  (b) grads == NULL: the caller has already added this micro-batch's gradient sums
+ *      into the S buffers (adloco_gram_sqnorm with accumulate_sum) and passes its
+ *      n_i in per_sample_sqnorm (dev [b_micro], required); only Q and the count move. */
+int adloco_accumulate(adloco_ctx* ctx, adloco_accum* acc, const void* grads, adloco_dtype dtype,
+                      int64_t b_micro, int64_t P, int64_t row_stride, float* per_sample_sqnorm, void* stream);
+
+/* One test on everything accumulated: N = sum_bufs ||S/b||^2,
+ * V = centred_ss/(b-ddof) when every micro-batch was materialised, otherwise
+ * V = (Q - b N)/(b - ddof); then the batch rule and switch plan. */
+int adloco_accum_finalize(adloco_ctx* ctx, adloco_accum* acc, const adloco_test_params* params,
+                          adloco_test_sums* sums_dev, adloco_test_result* result_dev,
+                          adloco_test_result* result_host, void* stream);
+
+/* ---- outer step ----------------------------------------------------------- */
+
+/* Last loop of Algorithm 3 for one trainer, fused in one pass:
+ *   d      = (1/K) sum_k (theta - theta_k)
+ *   v'     = momentum v + d
+ *   u      = d + momentum v' (nesterov != 0)  |  v'
+ *   theta' = theta - lr u
+ *   inst_params  HOST array of K dev pointers, each [P] in inst_dtype (F32 or BF16),
+ *                separate allocations allowed; 1 <= K <= 64
+ *   theta_in/out, mom_in/out  dev [P] float; out may be the same pointer as in
+ *                (exact aliasing only); instances must not overlap theta or mom
+ *   inst_writeback  HOST array of K dev pointers (may be NULL, entries may be NULL):
+ *                each receives theta' rounded to inst_dtype (Algorithm 3 resets every
+ *                worker to the trainer's parameters at the next outer step)
+ * fp32 arithmetic, the K differences summed in the order k = 0..K-1. */
+int adloco_outer_step(adloco_ctx* ctx, const void* const* inst_params, adloco_dtype inst_dtype, int32_t K,
+                      int64_t P, const float* theta_in, float* theta_out, const float* mom_in, float* mom_out,
+                      float lr, float momentum, int nesterov, void* const* inst_writeback, void* stream);
+
+/* Same update with every buffer in HOST memory (inst_params_host: K host
+ * pointers; theta_host and mom_host are updated in place): panels are staged
+ * through device buffers the library owns, copies overlapped with the kernel.
+ * Synchronous. */
+int adloco_outer_step_host(adloco_ctx* ctx, const void* const* inst_params_host, adloco_dtype inst_dtype,
+                           int32_t K, int64_t P, float* theta_host, float* mom_host, float lr, float momentum,
+                           int nesterov, void* stream);
+
+/* ---- trainer merge --------------------------------------------------------- */
+
+/* CheckMerge (Algorithm 1), host only: writes into merge_idx (host, capacity >= w)
+ * the indices of the w trainers with the smallest b_req (ties: lower index first)
+ * and returns their number; 0 when w == 0, k <= 1 or w > k; negative status on
+ * bad arguments. */
+int adloco_check_merge(const int64_t* b_req, int32_t k, int32_t w, int32_t* merge_idx);
+
+/* DoMerge (Algorithm 2): x_merge = sum_j b_j x_j / sum_j b_j over the K members
+ * (HOST array of dev pointers, [P] each in `dtype`; weights HOST int64 > 0),
+ * written to `out` (dev [P] in `dtype`; may be one of the members, exactly).
+ * *rep (host, may be NULL) receives the member with the largest weight (lowest
+ * index on ties), the trainer that is kept. 1 <= K <= 64. */
+int adloco_merge(adloco_ctx* ctx, const void* const* members, const int64_t* weights, adloco_dtype dtype,
+                 int32_t K, int64_t P, void* out, int32_t* rep, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADLOCO_H */

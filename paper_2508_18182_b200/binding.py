@@ -1,0 +1,314 @@
+"""ctypes binding of libadloco.so: the same entry points as include/adloco.h,
+taking torch tensors.  Argument marshalling only -- every step of the path runs
+in the CUDA kernels behind the C ABI.  There is no fallback: if the library is
+not built or no CUDA device is present, loading or the first call fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libadloco.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
+F32, BF16 = 0, 1
+FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN = 1, 2, 4, 8
+
+# every symbol that include/adloco.h declares
+EXPORTS = (
+    "adloco_create", "adloco_destroy", "adloco_status_string", "adloco_last_cuda_error", "adloco_launch_count",
+    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_gram_sqnorm",
+    "adloco_accum_create", "adloco_accum_reset", "adloco_accum_destroy", "adloco_accumulate",
+    "adloco_accum_finalize", "adloco_outer_step", "adloco_outer_step_host", "adloco_check_merge", "adloco_merge",
+)
+
+
+class TestParams(C.Structure):
+    __test__ = False
+    _fields_ = [("eta", C.c_double), ("ddof", C.c_int32), ("switch_n", C.c_int32),
+                ("b_cur", C.c_int64), ("b_max", C.c_int64), ("b_cap", C.c_int64)]
+
+
+class TestSums(C.Structure):
+    __test__ = False
+    _fields_ = [("sum_sqnorm", C.c_double), ("sum_sq_gsum", C.c_double), ("centred_ss", C.c_double),
+                ("batch_count", C.c_int64), ("has_centred", C.c_int32), ("device_status", C.c_int32)]
+
+
+class TestResult(C.Structure):
+    __test__ = False
+    _fields_ = [("sum_sqnorm", C.c_double), ("mean_sqnorm", C.c_double), ("variance", C.c_double),
+                ("stat", C.c_double), ("batch_count", C.c_int64), ("b_req", C.c_int64),
+                ("accum_steps", C.c_int64), ("b_micro", C.c_int64), ("flags", C.c_uint32),
+                ("device_status", C.c_int32)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class AdlocoError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(msg)
+        self.status = status
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads libadloco.so (built in-tree by paper_2508_18182_b200.build); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise OSError(f"{LIB_PATH} is not built: run `python -m paper_2508_18182_b200.build`")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+    sig = {
+        "adloco_create": (C.c_int, [C.POINTER(vp), C.c_int]),
+        "adloco_destroy": (C.c_int, [vp]),
+        "adloco_status_string": (C.c_char_p, [C.c_int]),
+        "adloco_last_cuda_error": (C.c_char_p, [vp]),
+        "adloco_launch_count": (i64, [vp]),
+        "adloco_norm_test": (C.c_int, [vp, vp, C.c_int, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp, vp, vp, vp]),
+        "adloco_test_decide": (C.c_int, [vp, vp, C.POINTER(TestParams), vp, vp, vp]),
+        "adloco_norm_test_host": (C.c_int, [vp, vp, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp]),
+        "adloco_gram_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
+        "adloco_accum_create": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), i32]),
+        "adloco_accum_reset": (C.c_int, [vp, vp, vp]),
+        "adloco_accum_destroy": (C.c_int, [vp]),
+        "adloco_accumulate": (C.c_int, [vp, vp, vp, C.c_int, i64, i64, i64, vp, vp]),
+        "adloco_accum_finalize": (C.c_int, [vp, vp, C.POINTER(TestParams), vp, vp, vp, vp]),
+        "adloco_outer_step": (C.c_int, [vp, C.POINTER(vp), C.c_int, i32, i64, vp, vp, vp, vp, f32, f32, C.c_int,
+                                        C.POINTER(vp), vp]),
+        "adloco_outer_step_host": (C.c_int, [vp, C.POINTER(vp), C.c_int, i32, i64, vp, vp, f32, f32, C.c_int, vp]),
+        "adloco_check_merge": (C.c_int, [C.POINTER(i64), i32, i32, C.POINTER(i32)]),
+        "adloco_merge": (C.c_int, [vp, C.POINTER(vp), C.POINTER(i64), C.c_int, i32, i64, vp, C.POINTER(i32), vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _dtype_code(dt):
+    if dt == torch.float32:
+        return F32
+    if dt == torch.bfloat16:
+        return BF16
+    raise AdlocoError(ERR_UNSUPPORTED, f"unsupported dtype {dt}")
+
+
+def make_params(eta, ddof=1, b_cur=1, b_max=1, b_cap=0, switch_n=2) -> TestParams:
+    return TestParams(float(eta), int(ddof), int(switch_n), int(b_cur), int(b_max), int(b_cap))
+
+
+class Context:
+    """One adloco_ctx on a CUDA device."""
+
+    def __init__(self, device: int = 0):
+        self.lib = load_library()
+        h = C.c_void_p()
+        rc = self.lib.adloco_create(C.byref(h), int(device))
+        if rc != OK:
+            raise AdlocoError(rc, f"adloco_create: {self.lib.adloco_status_string(rc).decode()}")
+        self.h = h
+        self.device = torch.device("cuda", int(device))
+        # small device/pinned scratch for results (torch owns the memory)
+        self._res_dev = torch.zeros(TestResult_size(), dtype=torch.uint8, device=self.device)
+        self._res_host = torch.zeros(TestResult_size(), dtype=torch.uint8).pin_memory()
+        self._sums_dev = torch.zeros(C.sizeof(TestSums), dtype=torch.uint8, device=self.device)
+
+    def close(self):
+        if getattr(self, "h", None):
+            torch.cuda.synchronize(self.device)
+            self.lib.adloco_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def check(self, rc: int, what: str):
+        if rc != OK:
+            msg = self.lib.adloco_status_string(rc).decode()
+            if rc == ERR_CUDA:
+                msg += ": " + self.lib.adloco_last_cuda_error(self.h).decode()
+            raise AdlocoError(rc, f"{what}: {msg}")
+
+    @property
+    def launch_count(self) -> int:
+        return int(self.lib.adloco_launch_count(self.h))
+
+    def _read_result(self, stream=None) -> TestResult:
+        (stream or torch.cuda.current_stream()).synchronize()
+        return TestResult.from_buffer_copy(self._res_host.numpy().tobytes())
+
+    def read_sums(self, sums_dev=None) -> TestSums:
+        t = self._sums_dev if sums_dev is None else sums_dev
+        return TestSums.from_buffer_copy(t.cpu().numpy().tobytes())
+
+    # ------------------------------------------------------------------ norm test
+    def norm_test(self, G, params: TestParams, *, per_sample_sqnorm=None, grad_sum=None, stream=None,
+                  sync=True):
+        """adloco_norm_test on a [B, P] float32 CUDA tensor (rows may be strided).
+        Returns the TestResult (after synchronising) or None when sync=False."""
+        B, P = G.shape
+        stride = G.stride(0) if B > 1 else max(G.stride(0), P)
+        if G.stride(1) != 1:
+            raise AdlocoError(ERR_INVALID_ARG, "columns must be contiguous")
+        rc = self.lib.adloco_norm_test(self.h, _ptr(G), _dtype_code(G.dtype), B, P, stride, C.byref(params),
+                                       _ptr(per_sample_sqnorm), _ptr(grad_sum), _ptr(self._sums_dev),
+                                       _ptr(self._res_dev), _ptr(self._res_host), _stream(stream))
+        self.check(rc, "adloco_norm_test")
+        return self._read_result(stream) if sync else None
+
+    def test_decide(self, params: TestParams, *, sums_dev=None, stream=None, sync=True):
+        """adloco_test_decide on the sums of the last norm_test (or the given device sums)."""
+        s = self._sums_dev if sums_dev is None else sums_dev
+        rc = self.lib.adloco_test_decide(self.h, _ptr(s), C.byref(params), _ptr(self._res_dev),
+                                         _ptr(self._res_host), _stream(stream))
+        self.check(rc, "adloco_test_decide")
+        return self._read_result(stream) if sync else None
+
+    def norm_test_host(self, G_host, params: TestParams, *, per_sample_sqnorm_host=None, stream=None):
+        """adloco_norm_test_host on a [B, P] float32 HOST tensor (ideally pinned)."""
+        B, P = G_host.shape
+        res = TestResult()
+        rc = self.lib.adloco_norm_test_host(self.h, _ptr(G_host), B, P, G_host.stride(0) if B > 1 else P,
+                                            C.byref(params), _ptr(per_sample_sqnorm_host),
+                                            C.cast(C.byref(res), C.c_void_p), _stream(stream))
+        self.check(rc, "adloco_norm_test_host")
+        return res
+
+    # ------------------------------------------------------------------ Gram path
+    def gram_sqnorm(self, X, D, per_sample_sqnorm, *, accumulate_norms=False, grad_sum=None,
+                    accumulate_sum=False, stream=None):
+        B, T, d_in = X.shape
+        d_out = D.shape[2]
+        if X.dtype != torch.bfloat16 or D.dtype != torch.bfloat16 or not X.is_contiguous() or not D.is_contiguous():
+            raise AdlocoError(ERR_INVALID_ARG, "X and D must be contiguous bfloat16")
+        rc = self.lib.adloco_gram_sqnorm(self.h, _ptr(X), _ptr(D), B, T, d_in, d_out, _ptr(per_sample_sqnorm),
+                                         int(accumulate_norms), _ptr(grad_sum), int(accumulate_sum),
+                                         _stream(stream))
+        self.check(rc, "adloco_gram_sqnorm")
+
+    # ------------------------------------------------------------------ outer step
+    def outer_step(self, instances, theta_in, mom_in, *, lr, momentum, nesterov=True, theta_out=None,
+                   mom_out=None, writeback=None, stream=None):
+        """adloco_outer_step; theta_out / mom_out default to in-place."""
+        K = len(instances)
+        P = theta_in.numel()
+        arr = (C.c_void_p * K)(*[t.data_ptr() for t in instances])
+        wb = None
+        if writeback is not None:
+            wb = (C.c_void_p * K)(*[(t.data_ptr() if t is not None else None) for t in writeback])
+        theta_out = theta_in if theta_out is None else theta_out
+        mom_out = mom_in if mom_out is None else mom_out
+        rc = self.lib.adloco_outer_step(self.h, arr, _dtype_code(instances[0].dtype), K, P, _ptr(theta_in),
+                                        _ptr(theta_out), _ptr(mom_in), _ptr(mom_out), float(lr), float(momentum),
+                                        int(bool(nesterov)), wb, _stream(stream))
+        self.check(rc, "adloco_outer_step")
+        return theta_out, mom_out
+
+    def outer_step_host(self, instances_host, theta_host, mom_host, *, lr, momentum, nesterov=True, stream=None):
+        K = len(instances_host)
+        arr = (C.c_void_p * K)(*[t.data_ptr() for t in instances_host])
+        rc = self.lib.adloco_outer_step_host(self.h, arr, _dtype_code(instances_host[0].dtype), K,
+                                             theta_host.numel(), _ptr(theta_host), _ptr(mom_host), float(lr),
+                                             float(momentum), int(bool(nesterov)), _stream(stream))
+        self.check(rc, "adloco_outer_step_host")
+
+    # ------------------------------------------------------------------ merge
+    def merge(self, members, weights, out, *, stream=None) -> int:
+        K = len(members)
+        arr = (C.c_void_p * K)(*[t.data_ptr() for t in members])
+        w = (C.c_int64 * K)(*[int(x) for x in weights])
+        rep = C.c_int32(-1)
+        rc = self.lib.adloco_merge(self.h, arr, w, _dtype_code(members[0].dtype), K, members[0].numel(),
+                                   _ptr(out), C.byref(rep), _stream(stream))
+        self.check(rc, "adloco_merge")
+        return rep.value
+
+
+def TestResult_size() -> int:
+    return C.sizeof(TestResult)
+
+
+def check_merge(b_req, w: int):
+    """adloco_check_merge (host only)."""
+    lib = load_library()
+    k = len(b_req)
+    arr = (C.c_int64 * max(k, 1))(*[int(x) for x in b_req])
+    out = (C.c_int32 * max(w, 1))()
+    n = lib.adloco_check_merge(arr, k, int(w), out)
+    if n < 0:
+        raise AdlocoError(n, "adloco_check_merge: " + lib.adloco_status_string(n).decode())
+    return [out[i] for i in range(n)]
+
+
+class Accumulator:
+    """adloco_accum over caller-owned float32 sum buffers (switch mode)."""
+
+    def __init__(self, ctx: Context, sum_bufs):
+        self.ctx = ctx
+        self.bufs = list(sum_bufs)
+        n = len(self.bufs)
+        ptrs = (C.c_void_p * n)(*[t.data_ptr() for t in self.bufs])
+        sizes = (C.c_int64 * n)(*[t.numel() for t in self.bufs])
+        h = C.c_void_p()
+        rc = ctx.lib.adloco_accum_create(ctx.h, C.byref(h), ptrs, sizes, n)
+        ctx.check(rc, "adloco_accum_create")
+        self.h = h
+
+    def reset(self, stream=None):
+        self.ctx.check(self.ctx.lib.adloco_accum_reset(self.ctx.h, self.h, _stream(stream)), "adloco_accum_reset")
+
+    def accumulate(self, G=None, *, per_sample_sqnorm=None, b_micro=None, stream=None):
+        if G is not None:
+            b, P = G.shape
+            stride = G.stride(0) if b > 1 else max(G.stride(0), P)
+            rc = self.ctx.lib.adloco_accumulate(self.ctx.h, self.h, _ptr(G), _dtype_code(G.dtype), b, P, stride,
+                                                _ptr(per_sample_sqnorm), _stream(stream))
+        else:
+            b = per_sample_sqnorm.numel() if b_micro is None else int(b_micro)
+            rc = self.ctx.lib.adloco_accumulate(self.ctx.h, self.h, None, F32, b, 0, 0,
+                                                _ptr(per_sample_sqnorm), _stream(stream))
+        self.ctx.check(rc, "adloco_accumulate")
+
+    def finalize(self, params: TestParams, *, stream=None, sync=True):
+        c = self.ctx
+        rc = c.lib.adloco_accum_finalize(c.h, self.h, C.byref(params), _ptr(c._sums_dev), _ptr(c._res_dev),
+                                         _ptr(c._res_host), _stream(stream))
+        c.check(rc, "adloco_accum_finalize")
+        return c._read_result(stream) if sync else None
+
+    def close(self):
+        if getattr(self, "h", None):
+            torch.cuda.synchronize(self.ctx.device)
+            self.ctx.lib.adloco_accum_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

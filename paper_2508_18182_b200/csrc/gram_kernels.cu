@@ -1,0 +1,510 @@
+// Tensor-core path (tcgen05 + TMEM + TMA) for linear layers:
+//
+//   gram_sqnorm_kernel  n_i = <X_i X_i^T, D_i D_i^T>_F, the squared Frobenius norm of
+//                       sample i's weight gradient D_i^T X_i, without forming it:
+//                       for every 128x128 tile (t, s >= t) of the token-by-token
+//                       Gram matrices both products are accumulated in TMEM and the
+//                       epilogue reduces their elementwise product.
+//   mean_grad_kernel    S (+)= sum_i D_i^T X_i, the batch gradient sum, a GEMM whose
+//                       contraction runs over all tokens of all samples.
+//
+// Both are persistent, warp-specialised kernels: warp 0 issues TMA tile loads
+// into a ring of shared-memory stages, warp 1 issues tcgen05.mma from shared
+// memory into TMEM accumulators (double-buffered), warps 2-5 drain the
+// accumulators.  Every wait is bounded; a wait that runs out raises a status
+// word and all roles leave through the common teardown.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace adloco {
+
+using namespace ptx;
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
+constexpr uint64_t kDrainLimitNs = 50000000ull;    // 50 ms per barrier while leaving after a time-out
+constexpr int TC_THREADS = 192;
+
+struct PipeState {
+    uint32_t stage = 0, phase = 0;
+    __device__ __forceinline__ void advance(uint32_t nstages) {
+        if (++stage == nstages) { stage = 0; phase ^= 1u; }
+    }
+};
+
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// =====================================================================================
+// Gram kernel
+// =====================================================================================
+constexpr int GR_TILE = 128;                       // tokens per tile side (M = N = 128)
+constexpr int GR_BK = 64;                          // features per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int GR_STAGES = 6;
+constexpr int GR_TILE_BYTES = GR_TILE * GR_BK * 2; // 16 KB
+constexpr int GR_STAGE_BYTES = 2 * GR_TILE_BYTES;  // t-tile and s-tile
+constexpr int GR_SMEM = GR_STAGES * GR_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+
+struct GramArgs {
+    int B, T, d_in, d_out;
+    int nt;           // token tiles per sample
+    int pairs;        // nt (nt + 1) / 2 tile pairs (s >= t)
+    int total_items;  // B * pairs
+    float* n;         // [B], += (zeroed by the launcher unless accumulating)
+    int* status;
+};
+
+__device__ __forceinline__ void gram_decode(int item, const GramArgs& a, int& i, int& ti, int& tj) {
+    i = item / a.pairs;
+    int p = item - i * a.pairs;
+    ti = 0;
+    while (p >= a.nt - ti) { p -= a.nt - ti; ++ti; }
+    tj = ti + p;
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
+                   const GramArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_base = smem_base + GR_STAGES * GR_STAGE_BYTES;
+    // barrier slots (8 bytes each): full[S], empty[S], tmem_full[2], tmem_empty[2], drain
+    auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (GR_STAGES + s); };
+    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * GR_STAGES + b); };
+    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * GR_STAGES + 2 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * GR_STAGES + 4);
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (uint32_t s = 0; s < GR_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        mbar_init(drain_bar, 1);
+        fence_barrier_init();
+        prefetch_tmap(&tmX);
+        prefetch_tmap(&tmD);
+    }
+    if (warp == 1) {  // TMEM: two buffers of (X X^T | D D^T) accumulators, 128 columns each
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    const int kx = (a.d_in + GR_BK - 1) / GR_BK, kd = (a.d_out + GR_BK - 1) / GR_BK;
+    const int chunks = kx + kd;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            PipeState ps;
+            uint32_t issued = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < a.total_items; item += gridDim.x) {
+                int i, ti, tj;
+                gram_decode(item, a, i, ti, tj);
+                const bool diag = (ti == tj);
+                for (int c = 0; c < chunks; ++c) {
+                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                    const bool is_x = c < kx;
+                    const CUtensorMap* map = is_x ? &tmX : &tmD;
+                    const int k0 = (is_x ? c : c - kx) * GR_BK;
+                    const uint32_t sA = smem_base + ps.stage * GR_STAGE_BYTES;
+                    mbar_arrive_expect_tx(full_bar(ps.stage), diag ? GR_TILE_BYTES : GR_STAGE_BYTES);
+                    tma_load_3d(sA, map, full_bar(ps.stage), k0, ti * GR_TILE, i);
+                    if (!diag) tma_load_3d(sA + GR_TILE_BYTES, map, full_bar(ps.stage), k0, tj * GR_TILE, i);
+                    ++issued;
+                    ps.advance(GR_STAGES);
+                }
+            }
+            if (!ok) {
+                // leaving after a time-out: let the copies still in flight land first
+                PipeState q = ps;
+                const uint32_t back = issued < GR_STAGES ? issued : GR_STAGES;
+                for (uint32_t r = 0; r < back; ++r) {
+                    if (q.stage == 0) { q.stage = GR_STAGES - 1; q.phase ^= 1u; } else { --q.stage; }
+                    int never = 0;
+                    mbar_wait(full_bar(q.stage), q.phase, &never, kDrainLimitNs);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(GR_TILE, GR_TILE, 0, 0);
+            PipeState ps;
+            bool ok = true;
+            int n_item = 0;
+            for (int item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++n_item) {
+                int i, ti, tj;
+                gram_decode(item, a, i, ti, tj);
+                const bool diag = (ti == tj);
+                const uint32_t buf = n_item & 1, use = n_item >> 1;
+                if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                tc_fence_after();
+                for (int c = 0; c < chunks; ++c) {
+                    if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, kWaitLimitNs)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t acc = tmem_base + buf * 256u + (c < kx ? 0u : 128u);
+                    const bool first = (c == 0 || c == kx);
+                    const uint32_t sA = smem_base + ps.stage * GR_STAGE_BYTES;
+                    const uint32_t sB = diag ? sA : sA + GR_TILE_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < GR_BK / 16; ++kk) {
+                        // K-major, 128-byte swizzle: rows of 128 B, 8-row groups 1024 B apart;
+                        // 16 features further along K = 32 bytes further in the row
+                        const uint64_t da = smem_desc_sw128(sA + kk * 32, 16, 1024);
+                        const uint64_t db = smem_desc_sw128(sB + kk * 32, 16, 1024);
+                        mma_bf16(acc, da, db, idesc, (first && kk == 0) ? 0u : 1u);
+                    }
+                    mma_commit(empty_bar(ps.stage));   // stage reusable once these MMAs have read it
+                    ps.advance(GR_STAGES);
+                }
+                if (ok) mma_commit(tfull_bar(buf));    // both accumulators of this item complete
+            }
+            if (!ok) {
+                mma_commit(drain_bar);
+                int never = 0;
+                mbar_wait(drain_bar, 0, &never, kDrainLimitNs);
+            }
+        }
+    } else {
+        // ---------------- epilogue: sum over the tile of (X X^T) .* (D D^T) ----------------
+        const uint32_t q = warp & 3;   // TMEM lanes 32q .. 32q+31 belong to this warp
+        int n_item = 0;
+        for (int item = blockIdx.x; item < a.total_items; item += gridDim.x, ++n_item) {
+            int i, ti, tj;
+            gram_decode(item, a, i, ti, tj);
+            const uint32_t buf = n_item & 1, use = n_item >> 1;
+            if (!mbar_wait(tfull_bar(buf), use & 1u, abortp, kWaitLimitNs)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + buf * 256u;
+            float sum = 0.f;
+#pragma unroll 1
+            for (int cc = 0; cc < GR_TILE / 32; ++cc) {
+                uint32_t x[32], d[32];
+                tmem_ld32(taddr + cc * 32, x);
+                tmem_ld32(taddr + 128 + cc * 32, d);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) sum = fmaf(__uint_as_float(x[e]), __uint_as_float(d[e]), sum);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            const float w = warp_sum_f(sum);
+            // tiles below the diagonal are never computed: an off-diagonal tile counts twice
+            if (lane == 0) atomicAdd(a.n + i, ti == tj ? w : 2.0f * w);
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
+}
+
+// =====================================================================================
+// mean-gradient kernel: S[d_out, d_in] += sum over samples and tokens of delta x^T
+// =====================================================================================
+constexpr int MG_BM = 128;                          // d_out rows per tile
+constexpr int MG_BN = 256;                          // d_in columns per tile
+constexpr int MG_BK = 64;                           // tokens per stage
+constexpr int MG_STAGES = 4;
+constexpr int MG_BOX_BYTES = 64 * MG_BK * 2;        // one TMA box: 64 features x 64 tokens = 8 KB
+constexpr int MG_A_BYTES = (MG_BM / 64) * MG_BOX_BYTES;
+constexpr int MG_B_BYTES = (MG_BN / 64) * MG_BOX_BYTES;
+constexpr int MG_STAGE_BYTES = MG_A_BYTES + MG_B_BYTES;   // 48 KB
+constexpr int MG_SMEM = MG_STAGES * MG_STAGE_BYTES + 1024 + 256;
+
+struct MeanGradArgs {
+    int B, T, d_in, d_out;
+    int ntm, ntn;       // tiles along d_out, d_in
+    int64_t units;      // ntm * ntn * B (tile-major, sample-minor)
+    float* S;           // [d_out, d_in], += (zeroed by the launcher unless accumulating)
+    int* status;
+};
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
+                 const MeanGradArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_base = smem_base + MG_STAGES * MG_STAGE_BYTES;
+    auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (MG_STAGES + s); };
+    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * MG_STAGES + b); };
+    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * MG_STAGES + 2 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * MG_STAGES + 4);
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (uint32_t s = 0; s < MG_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        mbar_init(drain_bar, 1);
+        fence_barrier_init();
+        prefetch_tmap(&tmX);
+        prefetch_tmap(&tmD);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);   // two 128x256 fp32 accumulators
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    // this CTA's contiguous share of the (tile, sample) units
+    const int64_t u0 = a.units * blockIdx.x / gridDim.x;
+    const int64_t u1 = a.units * (blockIdx.x + 1) / gridDim.x;
+    const int kt = (a.T + MG_BK - 1) / MG_BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            PipeState ps;
+            uint32_t issued = 0;
+            bool ok = true;
+            for (int64_t u = u0; ok && u < u1; ++u) {
+                const int tile = (int)(u / a.B), i = (int)(u % a.B);
+                const int tm = tile / a.ntn, tn = tile % a.ntn;
+                for (int c = 0; c < kt; ++c) {
+                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                    const uint32_t sA = smem_base + ps.stage * MG_STAGE_BYTES;
+                    const uint32_t sB = sA + MG_A_BYTES;
+                    mbar_arrive_expect_tx(full_bar(ps.stage), MG_STAGE_BYTES);
+#pragma unroll
+                    for (int mb = 0; mb < MG_BM / 64; ++mb)
+                        tma_load_3d(sA + mb * MG_BOX_BYTES, &tmD, full_bar(ps.stage), tm * MG_BM + mb * 64, c * MG_BK, i);
+#pragma unroll
+                    for (int nb = 0; nb < MG_BN / 64; ++nb)
+                        tma_load_3d(sB + nb * MG_BOX_BYTES, &tmX, full_bar(ps.stage), tn * MG_BN + nb * 64, c * MG_BK, i);
+                    ++issued;
+                    ps.advance(MG_STAGES);
+                }
+            }
+            if (!ok) {
+                PipeState q = ps;
+                const uint32_t back = issued < MG_STAGES ? issued : MG_STAGES;
+                for (uint32_t r = 0; r < back; ++r) {
+                    if (q.stage == 0) { q.stage = MG_STAGES - 1; q.phase ^= 1u; } else { --q.stage; }
+                    int never = 0;
+                    mbar_wait(full_bar(q.stage), q.phase, &never, kDrainLimitNs);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // both operands are stored with the contraction index (tokens) strided: MN-major
+            constexpr uint32_t idesc = idesc_bf16_f32(MG_BM, MG_BN, 1, 1);
+            PipeState ps;
+            bool ok = true;
+            int seg = 0;
+            int64_t u = u0;
+            while (ok && u < u1) {
+                const int tile = (int)(u / a.B);
+                int64_t u_end = (int64_t)(tile + 1) * a.B;     // end of this tile's samples
+                if (u_end > u1) u_end = u1;
+                const uint32_t buf = seg & 1, use = seg >> 1;
+                if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t acc = tmem_base + buf * 256u;
+                bool first = true;
+                for (; ok && u < u_end; ++u) {
+                    for (int c = 0; c < kt; ++c) {
+                        if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, kWaitLimitNs)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t sA = smem_base + ps.stage * MG_STAGE_BYTES;
+                        const uint32_t sB = sA + MG_A_BYTES;
+#pragma unroll
+                        for (int kk = 0; kk < MG_BK / 16; ++kk) {
+                            // MN-major, 128-byte swizzle: a token is a 128-byte row of 64 features,
+                            // 8-token groups 1024 B apart (stride offset), the next 64 features one
+                            // box further (leading offset); 16 tokens = 2 KB per MMA
+                            const uint64_t da = smem_desc_sw128(sA + kk * 2048, MG_BOX_BYTES, 1024);
+                            const uint64_t db = smem_desc_sw128(sB + kk * 2048, MG_BOX_BYTES, 1024);
+                            mma_bf16(acc, da, db, idesc, (first && kk == 0) ? 0u : 1u);
+                        }
+                        first = false;
+                        mma_commit(empty_bar(ps.stage));
+                        ps.advance(MG_STAGES);
+                    }
+                }
+                if (ok) mma_commit(tfull_bar(buf));
+                ++seg;
+            }
+            if (!ok) {
+                mma_commit(drain_bar);
+                int never = 0;
+                mbar_wait(drain_bar, 0, &never, kDrainLimitNs);
+            }
+        }
+    } else {
+        const uint32_t q = warp & 3;
+        int seg = 0;
+        int64_t u = u0;
+        while (u < u1) {
+            const int tile = (int)(u / a.B);
+            int64_t u_end = (int64_t)(tile + 1) * a.B;
+            if (u_end > u1) u_end = u1;
+            const int tm = tile / a.ntn, tn = tile % a.ntn;
+            const uint32_t buf = seg & 1, use = seg >> 1;
+            if (!mbar_wait(tfull_bar(buf), use & 1u, abortp, kWaitLimitNs)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + buf * 256u;
+            const int m = tm * MG_BM + (int)q * 32 + lane;
+            float* srow = a.S + (int64_t)m * a.d_in;
+#pragma unroll 1
+            for (int cc = 0; cc < MG_BN / 32; ++cc) {
+                uint32_t r[32];
+                tmem_ld32(taddr + cc * 32, r);
+                tmem_ld_wait();
+                const int n0 = tn * MG_BN + cc * 32;
+                if (m < a.d_out && n0 < a.d_in) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        const int n = n0 + e;
+                        if (n + 3 < a.d_in) {
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(srow + n),
+                                         "f"(__uint_as_float(r[e])), "f"(__uint_as_float(r[e + 1])),
+                                         "f"(__uint_as_float(r[e + 2])), "f"(__uint_as_float(r[e + 3]))
+                                         : "memory");
+                        } else {
+                            for (int z = 0; z < 4; ++z)
+                                if (n + z < a.d_in) atomicAdd(srow + n + z, __uint_as_float(r[e + z]));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            u = u_end;
+            ++seg;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
+}
+
+// =====================================================================================
+// host side
+// =====================================================================================
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn(adloco_ctx* ctx) {
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) {
+        set_cuda_error(ctx, e != cudaSuccess ? e : cudaErrorUnknown, "cuTensorMapEncodeTiled entry point");
+        return nullptr;
+    }
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+    return fn;
+}
+
+// bf16 tensor [B, T, d] (d contiguous) as a 3-D map {d, T, B} with a {64, box_tokens, 1}
+// box and 128-byte swizzle; out-of-range rows and columns read as zero.
+static int make_map(adloco_ctx* ctx, CUtensorMap* m, const void* base, int64_t B, int64_t T, int64_t d,
+                    uint32_t box_tokens) {
+    EncodeTiledFn fn = encode_fn(ctx);
+    if (!fn) return ADLOCO_ERR_CUDA;
+    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
+    const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)T * (cuuint64_t)d * 2};
+    const cuuint32_t box[3] = {64, box_tokens, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(ctx->cuda_err, sizeof(ctx->cuda_err), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return ADLOCO_ERR_CUDA;
+    }
+    return ADLOCO_OK;
+}
+
+int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                       int64_t d_out, float* n, int accumulate_norms, cudaStream_t st) {
+    CUtensorMap tmX, tmD;
+    int rc = make_map(ctx, &tmX, X, B, T, d_in, GR_TILE);
+    if (rc != ADLOCO_OK) return rc;
+    rc = make_map(ctx, &tmD, D, B, T, d_out, GR_TILE);
+    if (rc != ADLOCO_OK) return rc;
+    GramArgs a;
+    a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
+    a.nt = (int)((T + GR_TILE - 1) / GR_TILE);
+    const int64_t pairs = (int64_t)a.nt * (a.nt + 1) / 2;
+    if (pairs * B > 0x7fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    a.pairs = (int)pairs;
+    a.total_items = (int)(pairs * B);
+    a.n = n; a.status = ctx->gemm_status;
+    if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
+    static bool attr_set = false;
+    if (!attr_set) {
+        ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(gram_sqnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GR_SMEM));
+        attr_set = true;
+    }
+    const int grid = a.total_items < ctx->sm_count ? a.total_items : ctx->sm_count;
+    gram_sqnorm_kernel<<<grid, TC_THREADS, GR_SMEM, st>>>(tmX, tmD, a);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                     int64_t d_out, float* S, int accumulate_sum, cudaStream_t st) {
+    CUtensorMap tmX, tmD;
+    int rc = make_map(ctx, &tmX, X, B, T, d_in, MG_BK);
+    if (rc != ADLOCO_OK) return rc;
+    rc = make_map(ctx, &tmD, D, B, T, d_out, MG_BK);
+    if (rc != ADLOCO_OK) return rc;
+    MeanGradArgs a;
+    a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
+    a.ntm = (int)((d_out + MG_BM - 1) / MG_BM);
+    a.ntn = (int)((d_in + MG_BN - 1) / MG_BN);
+    a.units = (int64_t)a.ntm * a.ntn * B;
+    if (a.units / B > 0x7fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    a.S = S; a.status = ctx->gemm_status;
+    if (!accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
+    static bool attr_set = false;
+    if (!attr_set) {
+        ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(mean_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM));
+        attr_set = true;
+    }
+    const int grid = a.units < ctx->sm_count ? (int)a.units : ctx->sm_count;
+    mean_grad_kernel<<<grid, TC_THREADS, MG_SMEM, st>>>(tmX, tmD, a);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+void free_tmap_cache(adloco_ctx*) {}
+
+}  // namespace adloco

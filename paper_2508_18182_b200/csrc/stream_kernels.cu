@@ -1,0 +1,723 @@
+// HBM-streaming kernels: the one-pass norm test over materialised per-sample
+// gradients (also the switch-mode accumulation step), the batch rule, the fused
+// K-way pseudo-gradient average + momentum outer step, the weighted merge and
+// the squared-norm reduction over gradient-sum buffers.
+//
+// All of them move each input byte from HBM once with 128-bit accesses; the
+// arithmetic per byte is far below the machine balance, so grids are sized to
+// a multiple of the SM count and the only tuning that matters is bytes in
+// flight per SM.
+#include "common.cuh"
+
+namespace adloco {
+
+constexpr int NT_THREADS = 256;
+constexpr int NT_WARPS = NT_THREADS / 32;
+constexpr int NT_CHUNK = 8;  // rows loaded back to back before they are consumed
+
+// ---------------------------------------------------------------------------------
+// small device helpers
+// ---------------------------------------------------------------------------------
+__device__ __forceinline__ float4 ld_stream4(const float* p) {
+    return __ldcs(reinterpret_cast<const float4*>(p));
+}
+
+// up to four consecutive floats starting at p; lanes >= nvalid read as zero.
+// VEC = false is the path for rows that do not start on a 16-byte boundary.
+template <bool VEC = true>
+__device__ __forceinline__ float4 load4(const float* p, int nvalid) {
+    if (VEC && nvalid >= 4) return ld_stream4(p);
+    if (!VEC && nvalid >= 4) return make_float4(__ldcs(p), __ldcs(p + 1), __ldcs(p + 2), __ldcs(p + 3));
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (nvalid > 0) r.x = __ldcs(p);
+    if (nvalid > 1) r.y = __ldcs(p + 1);
+    if (nvalid > 2) r.z = __ldcs(p + 2);
+    return r;
+}
+
+template <bool VEC = true>
+__device__ __forceinline__ void store4(float* p, float4 v, int nvalid) {
+    if (VEC && nvalid >= 4) {
+        *reinterpret_cast<float4*>(p) = v;
+    } else if (nvalid >= 4) {
+        p[0] = v.x; p[1] = v.y; p[2] = v.z; p[3] = v.w;
+    } else {
+        if (nvalid > 0) p[0] = v.x;
+        if (nvalid > 1) p[1] = v.y;
+        if (nvalid > 2) p[2] = v.z;
+    }
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Sum of v over the block, fixed tree (deterministic); result valid in thread 0.
+__device__ double block_sum(double v, double* smem /* >= 32 doubles */) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) smem[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+    if (threadIdx.x == 0) {
+        const int nw = (blockDim.x + 31) >> 5;
+        for (int w = 0; w < nw; ++w) t += smem[w];
+    }
+    return t;
+}
+
+// Reduces RB per-row accumulators across the 32 lanes of a warp with a halving
+// exchange (about RB shuffles instead of 5*RB): at each step a lane keeps the
+// half of its values selected by one bit of its lane index and receives the
+// partner's sums for that half.
+template <int RB, int STEP>
+__device__ __forceinline__ void fold_step(float (&v)[RB], int lane) {
+    if constexpr (STEP < 5) {
+        constexpr int o = 16 >> STEP;
+        constexpr int c = RB >> STEP;  // values a lane still holds before this step
+        const bool upper = (lane & o) != 0;
+        if constexpr (c >= 2) {
+            constexpr int h = c / 2;
+#pragma unroll
+            for (int k = 0; k < h; ++k) {
+                const float send = upper ? v[k] : v[k + h];
+                const float keep = upper ? v[k + h] : v[k];
+                v[k] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+            }
+        } else {
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
+        }
+        fold_step<RB, STEP + 1>(v, lane);
+    }
+}
+
+// Adds the warp totals of the RB rows into dst[0..RB).  After the fold, lane l
+// holds rows l*RB/32 .. (RB >= 32), or row l/(32/RB) shared by 32/RB lanes.
+template <int RB>
+__device__ __forceinline__ void warp_rows_flush(float (&v)[RB], float* dst, int lane) {
+    fold_step<RB, 0>(v, lane);
+    if constexpr (RB >= 32) {
+        constexpr int per = RB / 32;
+#pragma unroll
+        for (int j = 0; j < per; ++j) dst[lane * per + j] += v[j];
+    } else {
+        constexpr int share = 32 / RB;
+        if ((lane % share) == 0) dst[lane / share] += v[0];
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// batch rule + switch plan (Section "Norm test", Section "Mode switching")
+// ---------------------------------------------------------------------------------
+__device__ void decide_device(const adloco_test_sums& s, const adloco_test_params& p, adloco_test_result* out) {
+    adloco_test_result r;
+    const int64_t b = s.batch_count;
+    const double bd = (double)b;
+    r.sum_sqnorm = s.sum_sqnorm;
+    r.mean_sqnorm = (b > 0) ? s.sum_sq_gsum / (bd * bd) : 0.0;
+    r.batch_count = b;
+    r.flags = 0;
+    r.device_status = s.device_status;
+    const int64_t i64max = 0x7fffffffffffffffLL;
+    if (b - p.ddof <= 0) {
+        r.flags |= ADLOCO_FLAG_UNDEFINED;
+        r.variance = 0.0;
+        r.stat = 0.0;
+        r.b_req = p.b_cur > 1 ? p.b_cur : 1;
+    } else {
+        const double denom = (double)(b - p.ddof);
+        r.variance = s.has_centred ? s.centred_ss / denom : (s.sum_sqnorm - bd * r.mean_sqnorm) / denom;
+        if (r.mean_sqnorm == 0.0) {
+            r.flags |= ADLOCO_FLAG_ZERO_MEAN;
+            r.stat = __longlong_as_double(0x7ff0000000000000LL);
+            r.b_req = p.b_cap > 0 ? p.b_cap : i64max;
+        } else {
+            r.stat = r.variance / (p.eta * p.eta * r.mean_sqnorm);
+            if (r.stat < 9.0e18) {
+                const int64_t c = (int64_t)ceil(r.stat);
+                r.b_req = c > 1 ? c : 1;
+            } else {
+                r.b_req = i64max;
+            }
+        }
+    }
+    if (p.b_cap > 0 && r.b_req > p.b_cap) r.b_req = p.b_cap;
+    if (r.b_req > p.b_cur) r.flags |= ADLOCO_FLAG_GROW;
+    // switch mode: accumulate only beyond switch_n * b_max (compare by division: no overflow)
+    if (r.b_req / p.b_max > p.switch_n || (r.b_req / p.b_max == p.switch_n && r.b_req % p.b_max != 0)) {
+        r.flags |= ADLOCO_FLAG_ACCUMULATE;
+        r.accum_steps = r.b_req / p.b_max + (r.b_req % p.b_max != 0 ? 1 : 0);
+        r.b_micro = p.b_max;
+    } else {
+        r.accum_steps = 1;
+        r.b_micro = r.b_req < p.b_max ? r.b_req : p.b_max;
+    }
+    *out = r;
+}
+
+__global__ void decide_kernel(const adloco_test_sums* sums, adloco_test_params p, adloco_test_result* out) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) decide_device(*sums, p, out);
+}
+
+// ---------------------------------------------------------------------------------
+// one-pass norm test
+// ---------------------------------------------------------------------------------
+struct NtArgs {
+    const float* G;
+    int64_t B, P, stride;
+    float* n_out;
+    float* S;
+    adloco_test_sums* sums;
+    adloco_test_result* result;
+    adloco_test_params params;
+    float* n_partials;
+    double* blk_scalars;
+    unsigned* ticket;
+    int mode, n_accum, first_panel, iters;
+};
+
+// Thread t of a block owns one group of four adjacent columns per iteration and
+// walks down all B rows of it: per column it keeps the sum and the sum of
+// squares of (G_ij - G_0j) -- shifting by the first row removes the mean before
+// squaring, so the centred sum of squares comes out without cancellation -- and
+// per row the running sum of squares (RB registers, rows tiled by RB).
+template <int RB, bool VEC>
+__global__ void __launch_bounds__(NT_THREADS, 2) norm_test_kernel(const __grid_constant__ NtArgs a) {
+    extern __shared__ float smem_rows[];  // [NT_WARPS][Bpad]
+    __shared__ double smem_red[32];
+    __shared__ int smem_is_last;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t B = a.B;
+    const int Bpad = (int)(((B + RB - 1) / RB) * RB);
+    for (int i = tid; i < NT_WARPS * Bpad; i += NT_THREADS) smem_rows[i] = 0.f;
+    __syncthreads();
+    float* my_rows = smem_rows + warp * Bpad;
+
+    const int64_t ngroups = (a.P + 3) >> 2;
+    const bool single_tile = (B <= RB);
+    const float Bf = (float)B;
+    const float invB = 1.0f / Bf;
+    // switch-mode accumulation: samples already accumulated before this micro-batch
+    const double c_prev_d = (a.mode == NT_MICRO) ? (double)a.sums->batch_count : 0.0;
+    const float inv_cprev = c_prev_d > 0.0 ? (float)(1.0 / c_prev_d) : 0.f;
+
+    float acc[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) acc[r] = 0.f;
+
+    double t_sumsq = 0.0, t_css = 0.0, t_chan = 0.0;
+    float f_sumsq = 0.f, f_css = 0.f, f_chan = 0.f;
+
+    for (int it = 0; it < a.iters; ++it) {
+        const int64_t g = ((int64_t)it * gridDim.x + blockIdx.x) * NT_THREADS + tid;
+        const int64_t col = g << 2;
+        int nvalid = 0;
+        if (g < ngroups) nvalid = (a.P - col) >= 4 ? 4 : (int)(a.P - col);
+        const float* rowp = a.G + (nvalid > 0 ? col : 0);
+
+        float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 sd = c, sdd = c;
+        for (int64_t i0 = 0; i0 < B; i0 += RB) {
+#pragma unroll
+            for (int r0 = 0; r0 < RB; r0 += NT_CHUNK) {
+                float4 x[NT_CHUNK];
+#pragma unroll
+                for (int u = 0; u < NT_CHUNK; ++u) {
+                    const bool ok = (i0 + r0 + u) < B;
+                    x[u] = load4<VEC>(rowp + (int64_t)(r0 + u) * a.stride, ok ? nvalid : 0);
+                }
+                if (i0 == 0 && r0 == 0) c = x[0];
+#pragma unroll
+                for (int u = 0; u < NT_CHUNK; ++u) {
+                    if ((i0 + r0 + u) < B) {
+                        const float4 v = x[u];
+                        float q = v.x * v.x;
+                        q = fmaf(v.y, v.y, q);
+                        q = fmaf(v.z, v.z, q);
+                        q = fmaf(v.w, v.w, q);
+                        acc[r0 + u] += q;
+                        const float dx = v.x - c.x, dy = v.y - c.y, dz = v.z - c.z, dw = v.w - c.w;
+                        sd.x += dx; sd.y += dy; sd.z += dz; sd.w += dw;
+                        sdd.x = fmaf(dx, dx, sdd.x); sdd.y = fmaf(dy, dy, sdd.y);
+                        sdd.z = fmaf(dz, dz, sdd.z); sdd.w = fmaf(dw, dw, sdd.w);
+                    }
+                }
+            }
+            rowp += (int64_t)RB * a.stride;
+            if (!single_tile) {
+                warp_rows_flush<RB>(acc, my_rows + i0, lane);
+#pragma unroll
+                for (int r = 0; r < RB; ++r) acc[r] = 0.f;
+            }
+        }
+
+        // per-column results of this group
+        float4 s;  // column sums over the B rows
+        s.x = fmaf(Bf, c.x, sd.x); s.y = fmaf(Bf, c.y, sd.y); s.z = fmaf(Bf, c.z, sd.z); s.w = fmaf(Bf, c.w, sd.w);
+        f_css += (sdd.x - sd.x * sd.x * invB) + (sdd.y - sd.y * sd.y * invB) +
+                 (sdd.z - sd.z * sd.z * invB) + (sdd.w - sd.w * sd.w * invB);
+        if (a.mode == NT_MICRO) {
+            float4 so = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (nvalid > 0) so = load4<VEC>(a.S + col, nvalid);
+            // pairwise (Chan) update of the centred sum of squares needs ||mean_mb - mean_prev||^2
+            const float ex = s.x * invB - so.x * inv_cprev, ey = s.y * invB - so.y * inv_cprev;
+            const float ez = s.z * invB - so.z * inv_cprev, ew = s.w * invB - so.w * inv_cprev;
+            f_chan += ex * ex + ey * ey + ez * ez + ew * ew;
+            s.x += so.x; s.y += so.y; s.z += so.z; s.w += so.w;
+            if (nvalid > 0) store4<VEC>(a.S + col, s, nvalid);
+        } else if (a.S != nullptr && nvalid > 0) {
+            store4<VEC>(a.S + col, s, nvalid);
+        }
+        f_sumsq += s.x * s.x + s.y * s.y + s.z * s.z + s.w * s.w;
+        if ((it & 15) == 15) {  // bound the length of the fp32 running sums
+            t_sumsq += (double)f_sumsq; t_css += (double)f_css; t_chan += (double)f_chan;
+            f_sumsq = f_css = f_chan = 0.f;
+        }
+    }
+    t_sumsq += (double)f_sumsq; t_css += (double)f_css; t_chan += (double)f_chan;
+    if (single_tile) warp_rows_flush<RB>(acc, my_rows, lane);
+
+    // block partials
+    const double b_sumsq = block_sum(t_sumsq, smem_red);
+    const double b_css = block_sum(t_css, smem_red);
+    const double b_chan = block_sum(t_chan, smem_red);
+    __syncthreads();
+    for (int64_t i = tid; i < B; i += NT_THREADS) {
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < NT_WARPS; ++w) t += smem_rows[w * Bpad + i];
+        a.n_partials[(int64_t)blockIdx.x * B + i] = t;
+    }
+    if (tid == 0) {
+        double* bs = a.blk_scalars + (int64_t)blockIdx.x * 4;
+        bs[0] = b_sumsq; bs[1] = b_css; bs[2] = b_chan;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned t = atomicAdd(a.ticket, 1u);
+        smem_is_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!smem_is_last) return;
+    __threadfence();
+
+    // last block: combine all partials in a fixed order, in fp64
+    double q_local = 0.0;
+    for (int64_t i = tid; i < B; i += NT_THREADS) {
+        double t = 0.0;
+        for (unsigned blk = 0; blk < gridDim.x; ++blk) t += (double)__ldcg(a.n_partials + (int64_t)blk * B + i);
+        if (a.n_out != nullptr) a.n_out[i] = a.n_accum ? a.n_out[i] + (float)t : (float)t;
+        q_local += t;
+    }
+    double p0 = 0.0, p1 = 0.0, p2 = 0.0;
+    for (unsigned blk = tid; blk < gridDim.x; blk += NT_THREADS) {
+        p0 += __ldcg(a.blk_scalars + (int64_t)blk * 4 + 0);
+        p1 += __ldcg(a.blk_scalars + (int64_t)blk * 4 + 1);
+        p2 += __ldcg(a.blk_scalars + (int64_t)blk * 4 + 2);
+    }
+    const double Q = block_sum(q_local, smem_red);
+    const double sumsq = block_sum(p0, smem_red);
+    const double css = block_sum(p1, smem_red);
+    const double chan = block_sum(p2, smem_red);
+    if (tid == 0) {
+        adloco_test_sums s = *a.sums;
+        if (a.mode == NT_ONESHOT || (a.mode == NT_PANEL && a.first_panel)) {
+            s.sum_sqnorm = Q; s.sum_sq_gsum = sumsq; s.centred_ss = css;
+            s.batch_count = B; s.has_centred = 1; s.device_status = 0;
+        } else if (a.mode == NT_PANEL) {
+            s.sum_sqnorm += Q; s.sum_sq_gsum += sumsq; s.centred_ss += css;
+        } else {  // NT_MICRO: rows are appended
+            const double cp = (double)s.batch_count, bb = (double)B;
+            s.centred_ss += css + (cp > 0.0 ? (cp * bb / (cp + bb)) * chan : 0.0);
+            s.sum_sqnorm += Q;
+            s.sum_sq_gsum = sumsq;  // ||S||^2 of the updated sum buffer
+            s.batch_count += B;
+        }
+        *a.sums = s;
+        if (a.result != nullptr) decide_device(s, a.params, a.result);
+        *a.ticket = 0u;
+    }
+}
+
+static int grow_workspace(adloco_ctx* ctx, size_t need_elems) {
+    if (need_elems <= ctx->n_partials_elems) return ADLOCO_OK;
+    if (ctx->n_partials) {
+        ADLOCO_CUDA_TRY(ctx, cudaDeviceSynchronize());
+        ADLOCO_CUDA_TRY(ctx, cudaFree(ctx->n_partials));
+        ctx->n_partials = nullptr;
+        ctx->n_partials_elems = 0;
+    }
+    ADLOCO_CUDA_TRY(ctx, cudaMalloc(&ctx->n_partials, need_elems * sizeof(float)));
+    ctx->n_partials_elems = need_elems;
+    return ADLOCO_OK;
+}
+
+template <int RB, bool VEC>
+static int launch_nt(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
+    const int64_t ngroups = (l.P + 3) / 4;
+    const int64_t tiles = (ngroups + NT_THREADS - 1) / NT_THREADS;
+    const int Bpad = (int)(((l.B + RB - 1) / RB) * RB);
+    const size_t smem = (size_t)NT_WARPS * Bpad * sizeof(float);
+    auto kern = norm_test_kernel<RB, VEC>;
+    if (smem > 48 * 1024) ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NT_THREADS, smem));
+    if (per_sm < 1) return ADLOCO_ERR_WORKSPACE;
+    int64_t max_grid = (int64_t)ctx->sm_count * per_sm;
+    if (max_grid > ctx->max_grid) max_grid = ctx->max_grid;
+    // equal work per block: iters passes over a grid that just covers the tiles
+    const int64_t iters = (tiles + max_grid - 1) / max_grid;
+    const int64_t grid = (tiles + iters - 1) / iters;
+    int rc = grow_workspace(ctx, (size_t)grid * (size_t)l.B);
+    if (rc != ADLOCO_OK) return rc;
+
+    NtArgs a;
+    a.G = l.G; a.B = l.B; a.P = l.P; a.stride = l.stride;
+    a.n_out = l.n_out; a.S = l.S; a.sums = l.sums; a.result = l.result; a.params = l.params;
+    a.n_partials = ctx->n_partials; a.blk_scalars = ctx->blk_scalars; a.ticket = ctx->ticket;
+    a.mode = l.mode; a.n_accum = l.n_accum; a.first_panel = l.first_panel; a.iters = (int)iters;
+    kern<<<(unsigned)grid, NT_THREADS, smem, st>>>(a);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+int launch_norm_test(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
+    // 128-bit accesses need every row (and S) to start on a 16-byte boundary
+    const bool vec = aligned16(l.G) && (l.B == 1 || (l.stride % 4) == 0) && (l.S == nullptr || aligned16(l.S));
+    if (vec) {
+        if (l.B <= 16) return launch_nt<16, true>(ctx, l, st);
+        if (l.B <= 32) return launch_nt<32, true>(ctx, l, st);
+        return launch_nt<64, true>(ctx, l, st);
+    }
+    if (l.B <= 16) return launch_nt<16, false>(ctx, l, st);
+    if (l.B <= 32) return launch_nt<32, false>(ctx, l, st);
+    return launch_nt<64, false>(ctx, l, st);
+}
+
+int launch_decide(adloco_ctx* ctx, const adloco_test_sums* sums, const adloco_test_params& p,
+                  adloco_test_result* result, cudaStream_t st) {
+    decide_kernel<<<1, 32, 0, st>>>(sums, p, result);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+// ---------------------------------------------------------------------------------
+// outer step: K-way pseudo-gradient average + momentum update, one pass
+// ---------------------------------------------------------------------------------
+struct OuterArgs {
+    const void* inst[kMaxInstances];
+    void* wb[kMaxInstances];
+    const float* th_in;
+    float* th_out;
+    const float* v_in;
+    float* v_out;
+    int64_t P;
+    double invK;
+    float lr, mu;
+    int K, nesterov;
+};
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&p);
+}
+
+// The K differences theta - theta_k are summed in fp64: each difference is then
+// exact and so is (to 2^-53) their sum, which cancels heavily when the instances
+// scatter around theta.  The update itself is carried in fp64 as well and each
+// output is rounded to fp32 once, so results sit within one rounding of the
+// exact update for the fp32 lr and momentum given.
+__device__ __forceinline__ void outer_update(float th, float v, double acc, const OuterArgs& a, float& th_new, float& v_new) {
+    const double d = acc * a.invK;
+    const double vn = fma((double)a.mu, (double)v, d);
+    const double u = a.nesterov ? fma((double)a.mu, vn, d) : vn;
+    v_new = (float)vn;
+    th_new = (float)fma(-(double)a.lr, u, (double)th);
+}
+
+template <bool BF16, bool WB>
+__global__ void __launch_bounds__(256) outer_step_kernel(const __grid_constant__ OuterArgs a) {
+    constexpr int VEC = BF16 ? 8 : 4;
+    const int64_t nvec = a.P / VEC;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
+        float th[VEC], v[VEC];
+        double acc[VEC], thd[VEC];
+        {
+            const float4* tp = reinterpret_cast<const float4*>(a.th_in) + i * (VEC / 4);
+            const float4* vp = reinterpret_cast<const float4*>(a.v_in) + i * (VEC / 4);
+#pragma unroll
+            for (int h = 0; h < VEC / 4; ++h) {
+                const float4 t = __ldcs(tp + h), w = __ldcs(vp + h);
+                th[4 * h] = t.x; th[4 * h + 1] = t.y; th[4 * h + 2] = t.z; th[4 * h + 3] = t.w;
+                v[4 * h] = w.x; v[4 * h + 1] = w.y; v[4 * h + 2] = w.z; v[4 * h + 3] = w.w;
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) { acc[e] = 0.0; thd[e] = (double)th[e]; }
+#pragma unroll 4
+        for (int k = 0; k < a.K; ++k) {
+            if (BF16) {
+                const uint4 x = __ldcs(reinterpret_cast<const uint4*>(a.inst[k]) + i);
+                acc[0] += thd[0] - (double)bf16_lo(x.x); acc[1] += thd[1] - (double)bf16_hi(x.x);
+                acc[2] += thd[2] - (double)bf16_lo(x.y); acc[3] += thd[3] - (double)bf16_hi(x.y);
+                acc[4 % VEC] += thd[4 % VEC] - (double)bf16_lo(x.z); acc[5 % VEC] += thd[5 % VEC] - (double)bf16_hi(x.z);
+                acc[6 % VEC] += thd[6 % VEC] - (double)bf16_lo(x.w); acc[7 % VEC] += thd[7 % VEC] - (double)bf16_hi(x.w);
+            } else {
+                const float4 x = __ldcs(reinterpret_cast<const float4*>(a.inst[k]) + i);
+                acc[0] += thd[0] - (double)x.x; acc[1] += thd[1] - (double)x.y; acc[2] += thd[2] - (double)x.z; acc[3] += thd[3] - (double)x.w;
+            }
+        }
+        float tn[VEC], vn[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) outer_update(th[e], v[e], acc[e], a, tn[e], vn[e]);
+        float4* to = reinterpret_cast<float4*>(a.th_out) + i * (VEC / 4);
+        float4* vo = reinterpret_cast<float4*>(a.v_out) + i * (VEC / 4);
+#pragma unroll
+        for (int h = 0; h < VEC / 4; ++h) {
+            __stcs(to + h, make_float4(tn[4 * h], tn[4 * h + 1], tn[4 * h + 2], tn[4 * h + 3]));
+            __stcs(vo + h, make_float4(vn[4 * h], vn[4 * h + 1], vn[4 * h + 2], vn[4 * h + 3]));
+        }
+        if (WB) {
+            for (int k = 0; k < a.K; ++k) {
+                if (a.wb[k] == nullptr) continue;
+                if (BF16) {
+                    uint4 o;
+                    o.x = pack_bf16(tn[0], tn[1]); o.y = pack_bf16(tn[2], tn[3]);
+                    o.z = pack_bf16(tn[4 % VEC], tn[5 % VEC]); o.w = pack_bf16(tn[6 % VEC], tn[7 % VEC]);
+                    reinterpret_cast<uint4*>(a.wb[k])[i] = o;
+                } else {
+                    reinterpret_cast<float4*>(a.wb[k])[i] = make_float4(tn[0], tn[1], tn[2], tn[3]);
+                }
+            }
+        }
+    }
+    // ragged tail (P not a multiple of the vector width): scalar, first block only
+    if (blockIdx.x == 0) {
+        for (int64_t j = nvec * VEC + threadIdx.x; j < a.P; j += blockDim.x) {
+            const float th = a.th_in[j], v = a.v_in[j];
+            double acc = 0.0;
+            for (int k = 0; k < a.K; ++k) {
+                float x;
+                if (BF16) x = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.inst[k])[j]);
+                else x = reinterpret_cast<const float*>(a.inst[k])[j];
+                acc += (double)th - (double)x;
+            }
+            float tn, vn;
+            outer_update(th, v, acc, a, tn, vn);
+            a.th_out[j] = tn;
+            a.v_out[j] = vn;
+            if (WB) {
+                for (int k = 0; k < a.K; ++k) {
+                    if (a.wb[k] == nullptr) continue;
+                    if (BF16) reinterpret_cast<__nv_bfloat16*>(a.wb[k])[j] = __float2bfloat16_rn(tn);
+                    else reinterpret_cast<float*>(a.wb[k])[j] = tn;
+                }
+            }
+        }
+    }
+}
+
+static unsigned elementwise_grid(const adloco_ctx* ctx, int64_t nvec, int threads, int blocks_per_sm) {
+    int64_t want = (nvec + threads - 1) / threads;
+    const int64_t cap = (int64_t)ctx->sm_count * blocks_per_sm;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    return (unsigned)want;
+}
+
+int launch_outer_step(adloco_ctx* ctx, const OuterLaunch& l, cudaStream_t st) {
+    OuterArgs a;
+    for (int k = 0; k < kMaxInstances; ++k) {
+        a.inst[k] = k < l.K ? l.inst[k] : nullptr;
+        a.wb[k] = (k < l.K && l.has_wb) ? l.wb[k] : nullptr;
+    }
+    a.th_in = l.th_in; a.th_out = l.th_out; a.v_in = l.v_in; a.v_out = l.v_out;
+    a.P = l.P; a.lr = l.lr; a.mu = l.mu; a.invK = 1.0 / (double)l.K; a.K = l.K; a.nesterov = l.nesterov;
+    const int vec = l.bf16 ? 8 : 4;
+    const unsigned grid = elementwise_grid(ctx, l.P / vec, 256, 8);
+    if (l.bf16) {
+        if (l.has_wb) outer_step_kernel<true, true><<<grid, 256, 0, st>>>(a);
+        else outer_step_kernel<true, false><<<grid, 256, 0, st>>>(a);
+    } else {
+        if (l.has_wb) outer_step_kernel<false, true><<<grid, 256, 0, st>>>(a);
+        else outer_step_kernel<false, false><<<grid, 256, 0, st>>>(a);
+    }
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+// ---------------------------------------------------------------------------------
+// weighted merge of trainers (Algorithm 2): out = sum_k coef_k x_k
+// ---------------------------------------------------------------------------------
+struct MergeArgs {
+    const void* x[kMaxInstances];
+    float coef[kMaxInstances];
+    void* out;
+    int64_t P;
+    int K;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ MergeArgs a) {
+    constexpr int VEC = BF16 ? 8 : 4;
+    const int64_t nvec = a.P / VEC;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
+        float acc[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < a.K; ++k) {
+            const float w = a.coef[k];
+            if (BF16) {
+                const uint4 x = __ldcs(reinterpret_cast<const uint4*>(a.x[k]) + i);
+                acc[0] = fmaf(w, bf16_lo(x.x), acc[0]); acc[1] = fmaf(w, bf16_hi(x.x), acc[1]);
+                acc[2] = fmaf(w, bf16_lo(x.y), acc[2]); acc[3] = fmaf(w, bf16_hi(x.y), acc[3]);
+                acc[4 % VEC] = fmaf(w, bf16_lo(x.z), acc[4 % VEC]); acc[5 % VEC] = fmaf(w, bf16_hi(x.z), acc[5 % VEC]);
+                acc[6 % VEC] = fmaf(w, bf16_lo(x.w), acc[6 % VEC]); acc[7 % VEC] = fmaf(w, bf16_hi(x.w), acc[7 % VEC]);
+            } else {
+                const float4 x = __ldcs(reinterpret_cast<const float4*>(a.x[k]) + i);
+                acc[0] = fmaf(w, x.x, acc[0]); acc[1] = fmaf(w, x.y, acc[1]);
+                acc[2] = fmaf(w, x.z, acc[2]); acc[3] = fmaf(w, x.w, acc[3]);
+            }
+        }
+        if (BF16) {
+            uint4 o;
+            o.x = pack_bf16(acc[0], acc[1]); o.y = pack_bf16(acc[2], acc[3]);
+            o.z = pack_bf16(acc[4 % VEC], acc[5 % VEC]); o.w = pack_bf16(acc[6 % VEC], acc[7 % VEC]);
+            reinterpret_cast<uint4*>(a.out)[i] = o;
+        } else {
+            reinterpret_cast<float4*>(a.out)[i] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        }
+    }
+    if (blockIdx.x == 0) {
+        for (int64_t j = nvec * VEC + threadIdx.x; j < a.P; j += blockDim.x) {
+            float acc = 0.f;
+            for (int k = 0; k < a.K; ++k) {
+                float x;
+                if (BF16) x = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.x[k])[j]);
+                else x = reinterpret_cast<const float*>(a.x[k])[j];
+                acc = fmaf(a.coef[k], x, acc);
+            }
+            if (BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[j] = __float2bfloat16_rn(acc);
+            else reinterpret_cast<float*>(a.out)[j] = acc;
+        }
+    }
+}
+
+int launch_merge(adloco_ctx* ctx, const MergeLaunch& l, cudaStream_t st) {
+    MergeArgs a;
+    for (int k = 0; k < kMaxInstances; ++k) {
+        a.x[k] = k < l.K ? l.x[k] : nullptr;
+        a.coef[k] = k < l.K ? l.coef[k] : 0.f;
+    }
+    a.out = l.out; a.P = l.P; a.K = l.K;
+    const int vec = l.bf16 ? 8 : 4;
+    const unsigned grid = elementwise_grid(ctx, l.P / vec, 256, 8);
+    if (l.bf16) merge_kernel<true><<<grid, 256, 0, st>>>(a);
+    else merge_kernel<false><<<grid, 256, 0, st>>>(a);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+// ---------------------------------------------------------------------------------
+// accumulator helpers for the tensor-core path
+// ---------------------------------------------------------------------------------
+// Q += sum(n[0..b)), count += b; the centred sum is no longer available.
+__global__ void accum_add_norms_kernel(adloco_test_sums* state, const float* n, int64_t b) {
+    __shared__ double red[32];
+    double t = 0.0;
+    for (int64_t i = threadIdx.x; i < b; i += blockDim.x) t += (double)n[i];
+    const double tot = block_sum(t, red);
+    if (threadIdx.x == 0) {
+        state->sum_sqnorm += tot;
+        state->batch_count += b;
+        state->has_centred = 0;
+    }
+}
+
+int launch_accum_add_norms(adloco_ctx* ctx, adloco_accum* acc, const float* n, int64_t b, cudaStream_t st) {
+    accum_add_norms_kernel<<<1, 256, 0, st>>>(acc->state, n, b);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+constexpr int SQ_CHUNK = 4096;  // elements per block-iteration: 256 threads x 4 float4
+
+// ||S||^2 summed over all buffers of the accumulator -> state->sum_sq_gsum.
+__global__ void __launch_bounds__(256) accum_sqnorm_kernel(float* const* bufs, const int64_t* sizes,
+                                                           const int64_t* chunk_prefix, int n_bufs,
+                                                           int64_t total_chunks, double* blk_scalars,
+                                                           unsigned* ticket, adloco_test_sums* state) {
+    __shared__ double red[32];
+    __shared__ int is_last;
+    float f = 0.f;
+    double t = 0.0;
+    int since = 0;
+    for (int64_t ch = blockIdx.x; ch < total_chunks; ch += gridDim.x) {
+        // which buffer holds chunk ch: largest b with chunk_prefix[b] <= ch
+        int lo = 0, hi = n_bufs - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (chunk_prefix[mid] <= ch) lo = mid; else hi = mid - 1;
+        }
+        const float* base = bufs[lo];
+        const int64_t size = sizes[lo];
+        const int64_t off = (ch - chunk_prefix[lo]) * SQ_CHUNK;
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const int64_t j = off + ((int64_t)h * 256 + threadIdx.x) * 4;
+            if (j < size) {
+                const int nv = (size - j) >= 4 ? 4 : (int)(size - j);
+                const float4 x = load4(base + j, nv);
+                f += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+            }
+        }
+        if (++since == 16) { t += (double)f; f = 0.f; since = 0; }
+    }
+    t += (double)f;
+    const double b = block_sum(t, red);
+    if (threadIdx.x == 0) blk_scalars[(int64_t)blockIdx.x * 4] = b;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double p = 0.0;
+    for (unsigned blk = threadIdx.x; blk < gridDim.x; blk += blockDim.x) p += __ldcg(blk_scalars + (int64_t)blk * 4);
+    const double tot = block_sum(p, red);
+    if (threadIdx.x == 0) {
+        state->sum_sq_gsum = tot;
+        *ticket = 0u;
+    }
+}
+
+int launch_accum_sqnorm(adloco_ctx* ctx, adloco_accum* acc, cudaStream_t st) {
+    int64_t grid = acc->total_chunks;
+    const int64_t cap = (int64_t)ctx->sm_count * 8;
+    if (grid > cap) grid = cap;
+    if (grid > ctx->max_grid) grid = ctx->max_grid;
+    if (grid < 1) grid = 1;
+    accum_sqnorm_kernel<<<(unsigned)grid, 256, 0, st>>>(acc->bufs_dev, acc->sizes_dev, acc->chunk_prefix_dev,
+                                                       acc->n_bufs, acc->total_chunks, ctx->blk_scalars,
+                                                       ctx->ticket, acc->state);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+}  // namespace adloco

@@ -1,0 +1,110 @@
+"""GPU parity: adloco_gram_sqnorm (Gram-identity per-sample norms and the
+mean-gradient GEMM on the tensor cores) against the fp64 oracle, which forms
+every per-sample weight gradient explicitly."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle.adloco_oracle as O
+from paper_2508_18182_b200 import binding as A
+from paper_2508_18182_b200 import workloads as W
+from parity import TOL_BF16, assert_test_result
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = A.Context(0)
+    yield c
+    c.close()
+
+
+def _gpu_layer(ctx, X, D, want_S=True):
+    B = X.shape[0]
+    n = torch.full((B,), -5.0, device=DEV)
+    S = torch.full((D.shape[2], X.shape[2]), -5.0, device=DEV) if want_S else None
+    ctx.gram_sqnorm(X, D, n, grad_sum=S)
+    torch.cuda.synchronize()
+    return n, S
+
+
+def test_small_integer_layer_is_exact(ctx):
+    # every product and partial sum is an integer below 2^24: the result must be exact
+    X, D = W.small_integer_layer(3, 5, 8, 16, seed=9, device=DEV)
+    n, S = _gpu_layer(ctx, X, D)
+    n_ref, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
+    assert np.array_equal(n.cpu().numpy().astype(np.float64), n_ref)
+    assert np.array_equal(S.cpu().numpy().astype(np.float64), S_ref)
+
+
+@pytest.mark.parametrize("B,T,d_in,d_out", [
+    (2, 128, 64, 64),        # one tile, one chunk
+    (3, 256, 128, 192),      # off-diagonal tiles, several chunks
+    (2, 200, 72, 40),        # ragged T (not a multiple of 128 or 64), ragged d (multiples of 8 only)
+    (5, 1, 8, 8),            # a single token: n_i = |x|^2 |delta|^2
+    (1, 384, 768, 256),      # 3x3 token tiles, 12 + 4 chunks: the ring wraps
+    (4, 130, 264, 520),      # d_in > 256 and d_out > 512: several output tiles, ragged
+    (33, 64, 32, 48),
+])
+def test_layer_matches_oracle(ctx, B, T, d_in, d_out):
+    X, D = W.linear_layer(B, T, d_in, d_out, seed=B + T, device=DEV)
+    n, S = _gpu_layer(ctx, X, D)
+    n_ref, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
+    assert np.allclose(n.cpu().numpy(), n_ref, rtol=TOL_BF16, atol=0), (n.cpu().numpy() / n_ref)
+    scale = np.abs(S_ref).max()
+    assert np.allclose(S.cpu().numpy(), S_ref, rtol=TOL_BF16, atol=TOL_BF16 * scale * 0.05)
+    if T == 1:
+        x2 = (X.double() ** 2).sum((1, 2)).cpu().numpy()
+        d2 = (D.double() ** 2).sum((1, 2)).cpu().numpy()
+        assert np.allclose(n.cpu().numpy(), x2 * d2, rtol=1e-5)
+
+
+def test_accumulate_flags_and_unsupported_shapes(ctx):
+    X, D = W.linear_layer(2, 96, 64, 64, seed=1, device=DEV)
+    n, S = _gpu_layer(ctx, X, D)
+    n2, S2 = n.clone(), S.clone()
+    ctx.gram_sqnorm(X, D, n2, accumulate_norms=True, grad_sum=S2, accumulate_sum=True)
+    torch.cuda.synchronize()
+    assert torch.allclose(n2, 2 * n, rtol=1e-6) and torch.allclose(S2, 2 * S, rtol=1e-6, atol=1e-9)
+    # without the sum buffer only the norms are computed
+    n3 = torch.zeros(2, device=DEV)
+    ctx.gram_sqnorm(X, D, n3)
+    torch.cuda.synchronize()
+    assert torch.equal(n3, n)
+    Xb, Db = W.linear_layer(2, 16, 12, 64, seed=1, device=DEV)      # d_in not a multiple of 8
+    before = ctx.launch_count
+    with pytest.raises(A.AdlocoError) as e:
+        ctx.gram_sqnorm(Xb, Db, n3)
+    assert e.value.status == A.ERR_UNSUPPORTED and ctx.launch_count == before
+
+
+def test_whole_model_switch_mode_small(ctx):
+    """Two blocks of four linear layers, a batch of 12 processed as 3 accumulated
+    micro-batches of 4: per-sample norms accumulate across layers, gradient sums
+    across micro-batches, one test at the end."""
+    shapes = [(64, 192), (64, 64), (64, 256), (256, 64)] * 2
+    n_micro, b, T = 3, 4, 160
+    data = [[W.linear_layer(b, T, di, do, seed=1000 * j + l, device=DEV) for l, (di, do) in enumerate(shapes)]
+            for j in range(n_micro)]
+    sums = [torch.empty(do, di, device=DEV) for di, do in shapes]
+    acc = A.Accumulator(ctx, sums)
+    acc.reset()
+    n_mb = torch.zeros(b, device=DEV)
+    for j in range(n_micro):
+        for l, (X, D) in enumerate(data[j]):
+            ctx.gram_sqnorm(X, D, n_mb, accumulate_norms=(l > 0), grad_sum=sums[l], accumulate_sum=True)
+        acc.accumulate(per_sample_sqnorm=n_mb)
+    p = A.make_params(0.5, b_cur=12, b_max=4)
+    r = acc.finalize(p)
+    layers = [(np.concatenate([W.to_numpy(data[j][l][0]) for j in range(n_micro)]),
+               np.concatenate([W.to_numpy(data[j][l][1]) for j in range(n_micro)])) for l in range(len(shapes))]
+    ora = O.linear_layers_norm_test(layers, eta=0.5, b_cur=12, b_max=4, two_pass=True)
+    # V comes from Q - b N here: scale the tolerance by the cancellation it suffers
+    kappa = ora.sum_sqnorm / (ora.variance * 11)
+    assert_test_result(r, ora, p, TOL_BF16, stat_tol=TOL_BF16 * max(1.0, kappa), what="whole model")
+    assert r.flags & A.FLAG_ACCUMULATE
+    acc.close()
