@@ -151,6 +151,26 @@ int adloco_norm_test_host(adloco_ctx* ctx, const float* grads_host, int64_t B, i
                           const adloco_test_params* params, float* per_sample_sqnorm_host,
                           adloco_test_result* result_host, void* stream);
 
+/* Norm test for callers that must not allocate.  The paper has no counterpart:
+ * this is adloco_norm_test (same kernel, same results) with the reduction
+ * scratch in a device array built into the library (about 290 KB per GPU, held
+ * from library load to process exit) instead of an adloco_ctx, for callers that
+ * cannot call cudaMalloc where the test runs -- e.g. inside a step whose
+ * allocator pool is frozen, or with the device-memory budget already spent.
+ * It calls no cudaMalloc/cudaFree and no allocating library routine.
+ *   - runs on the CURRENT device, on `stream`; grads/per_sample_sqnorm (may be
+ *     NULL)/result_dev are caller-owned dev memory, result_host (may be NULL) is
+ *     filled by an async copy as in adloco_norm_test
+ *   - limit: B <= 64 rows (ADLOCO_ERR_UNSUPPORTED beyond); any P >= 1
+ *   - the first call on each device looks up the array's device address; make
+ *     that first call before any stream capture
+ *   - every call shares the one array: calls that overlap on the GPU (different
+ *     streams, or different threads) race and give wrong results; calls on one
+ *     stream are safe back to back. */
+int adloco_norm_test_noalloc(const float* grads, int64_t B, int64_t P, int64_t row_stride,
+                             const adloco_test_params* params, float* per_sample_sqnorm,
+                             adloco_test_result* result_dev, adloco_test_result* result_host, void* stream);
+
 /* ---- per-sample norms of a linear layer via the Gram identity ------------ */
 
 /* For a linear layer y = W x and a batch of B sequences of T tokens, sample i

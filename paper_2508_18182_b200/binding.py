@@ -22,7 +22,7 @@ FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN = 1, 2, 4, 8
 # every symbol that include/adloco.h declares
 EXPORTS = (
     "adloco_create", "adloco_destroy", "adloco_status_string", "adloco_last_cuda_error", "adloco_launch_count",
-    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_gram_sqnorm",
+    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_gram_sqnorm",
     "adloco_accum_create", "adloco_accum_reset", "adloco_accum_destroy", "adloco_accumulate",
     "adloco_accum_finalize", "adloco_outer_step", "adloco_outer_step_host", "adloco_check_merge", "adloco_merge",
 )
@@ -78,6 +78,7 @@ def load_library() -> C.CDLL:
         "adloco_norm_test": (C.c_int, [vp, vp, C.c_int, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp, vp, vp, vp]),
         "adloco_test_decide": (C.c_int, [vp, vp, C.POINTER(TestParams), vp, vp, vp]),
         "adloco_norm_test_host": (C.c_int, [vp, vp, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp]),
+        "adloco_norm_test_noalloc": (C.c_int, [vp, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp, vp]),
         "adloco_gram_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
         "adloco_accum_create": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), i32]),
         "adloco_accum_reset": (C.c_int, [vp, vp, vp]),
@@ -247,6 +248,22 @@ class Context:
                                    _ptr(out), C.byref(rep), _stream(stream))
         self.check(rc, "adloco_merge")
         return rep.value
+
+
+def norm_test_noalloc(G, params: TestParams, result_dev, result_host, *, per_sample_sqnorm=None, stream=None):
+    """adloco_norm_test_noalloc on the current device: no context, and nothing
+    is allocated by the library.  `result_dev` (device) and `result_host`
+    (pinned host) are uint8 tensors of at least sizeof(TestResult) bytes that the
+    caller owns.  Returns the TestResult after synchronising the stream."""
+    lib = load_library()
+    B, P = G.shape
+    stride = G.stride(0) if B > 1 else max(G.stride(0), P)
+    rc = lib.adloco_norm_test_noalloc(_ptr(G), B, P, stride, C.byref(params), _ptr(per_sample_sqnorm),
+                                      _ptr(result_dev), _ptr(result_host), _stream(stream))
+    if rc != OK:
+        raise AdlocoError(rc, "adloco_norm_test_noalloc: " + lib.adloco_status_string(rc).decode())
+    (stream or torch.cuda.current_stream()).synchronize()
+    return TestResult.from_buffer_copy(result_host.numpy().tobytes()[:C.sizeof(TestResult)])
 
 
 def TestResult_size() -> int:

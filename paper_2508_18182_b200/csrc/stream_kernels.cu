@@ -409,6 +409,112 @@ int launch_decide(adloco_ctx* ctx, const adloco_test_sums* sums, const adloco_te
 }
 
 // ---------------------------------------------------------------------------------
+// norm test without any allocation
+// ---------------------------------------------------------------------------------
+// Some callers cannot allocate device memory at the point where they need the
+// test: a training step whose caching-allocator pool is frozen for the step, or
+// a process that was handed a fixed device-memory budget and has spent it.  For them the reduction
+// scratch of the norm test (per-block partial row sums, per-block scalars, the
+// ticket counter and the sums record) lives in this file-scope device array
+// instead of a context's workspace.  Every GPU that loads the library holds
+// these bytes until the process exits.
+constexpr int NA_MAX_ROWS = 64;      // largest B the entry point accepts
+constexpr int NA_MAX_GRID = 1024;    // most blocks it ever launches
+constexpr size_t NA_PARTIALS_BYTES = (size_t)NA_MAX_GRID * NA_MAX_ROWS * sizeof(float);   // 256 KB
+constexpr size_t NA_SCALARS_BYTES = (size_t)NA_MAX_GRID * 4 * sizeof(double);             // 32 KB
+constexpr size_t NA_TAIL_BYTES = 512;                                                      // ticket + sums
+constexpr size_t NA_SCRATCH_BYTES = NA_PARTIALS_BYTES + NA_SCALARS_BYTES + NA_TAIL_BYTES;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NA_SCRATCH_BYTES];
+
+constexpr int NA_MAX_DEVICES = 64;
+static void* g_noalloc_ptr[NA_MAX_DEVICES];   // device address of the array, per device; nullptr until set up
+static int g_noalloc_sms[NA_MAX_DEVICES];
+
+}  // namespace adloco
+
+#include <mutex>
+
+namespace adloco {
+static std::mutex g_noalloc_mutex;
+
+template <int RB, bool VEC>
+static cudaError_t launch_nt_noalloc(const NtArgs& proto, int sm_count, cudaStream_t st) {
+    NtArgs a = proto;
+    const int64_t ngroups = (a.P + 3) / 4;
+    const int64_t tiles = (ngroups + NT_THREADS - 1) / NT_THREADS;
+    const int Bpad = (int)(((a.B + RB - 1) / RB) * RB);
+    const size_t smem = (size_t)NT_WARPS * Bpad * sizeof(float);   // at most 2 KB here
+    int64_t max_grid = (int64_t)sm_count * 2;
+    if (max_grid > NA_MAX_GRID) max_grid = NA_MAX_GRID;
+    const int64_t iters = (tiles + max_grid - 1) / max_grid;
+    const int64_t grid = (tiles + iters - 1) / iters;
+    a.iters = (int)iters;
+    norm_test_kernel<RB, VEC><<<(unsigned)grid, NT_THREADS, smem, st>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace adloco
+
+extern "C" __attribute__((visibility("default")))
+int adloco_norm_test_noalloc(const float* grads, int64_t B, int64_t P, int64_t row_stride,
+                             const adloco_test_params* params, float* per_sample_sqnorm,
+                             adloco_test_result* result_dev, adloco_test_result* result_host, void* stream) {
+    using namespace adloco;
+    if (!grads || !result_dev || B < 1 || P < 1 || row_stride < P) return ADLOCO_ERR_INVALID_ARG;
+    int rc = check_params(params);
+    if (rc != ADLOCO_OK) return rc;
+    if (B > NA_MAX_ROWS) return ADLOCO_ERR_UNSUPPORTED;   // the static scratch holds 64 rows per block
+    if ((reinterpret_cast<uintptr_t>(grads) & 3u) != 0) return ADLOCO_ERR_ALIGNMENT;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NA_MAX_DEVICES) return ADLOCO_ERR_CUDA;
+    {
+        // once per device, with that device current: the array's name is only a
+        // host-side handle, the kernel needs the address the runtime maps it to
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (g_noalloc_ptr[dev] == nullptr) {
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return ADLOCO_ERR_CUDA;
+            int sms = 0;
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+                return ADLOCO_ERR_CUDA;
+            g_noalloc_sms[dev] = sms;
+            g_noalloc_ptr[dev] = ptr;
+        }
+    }
+    unsigned char* base = static_cast<unsigned char*>(g_noalloc_ptr[dev]);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    NtArgs a;
+    a.G = grads; a.B = B; a.P = P; a.stride = row_stride;
+    a.n_out = per_sample_sqnorm; a.S = nullptr;
+    a.n_partials = reinterpret_cast<float*>(base);
+    a.blk_scalars = reinterpret_cast<double*>(base + NA_PARTIALS_BYTES);
+    a.ticket = reinterpret_cast<unsigned*>(base + NA_PARTIALS_BYTES + NA_SCALARS_BYTES);
+    a.sums = reinterpret_cast<adloco_test_sums*>(base + NA_PARTIALS_BYTES + NA_SCALARS_BYTES + 256);
+    a.result = result_dev; a.params = *params;
+    a.mode = NT_ONESHOT; a.n_accum = 0; a.first_panel = 1; a.iters = 0;
+    // the array keeps whatever the last call left: the ticket must start at zero
+    if (cudaMemsetAsync(a.ticket, 0, NA_TAIL_BYTES, st) != cudaSuccess) return ADLOCO_ERR_CUDA;
+    const bool vec = aligned16(grads) && (B == 1 || (row_stride % 4) == 0);
+    cudaError_t e;
+    const int sms = g_noalloc_sms[dev];
+    if (vec) {
+        e = B <= 16 ? launch_nt_noalloc<16, true>(a, sms, st)
+          : B <= 32 ? launch_nt_noalloc<32, true>(a, sms, st) : launch_nt_noalloc<64, true>(a, sms, st);
+    } else {
+        e = B <= 16 ? launch_nt_noalloc<16, false>(a, sms, st)
+          : B <= 32 ? launch_nt_noalloc<32, false>(a, sms, st) : launch_nt_noalloc<64, false>(a, sms, st);
+    }
+    if (e != cudaSuccess) return ADLOCO_ERR_CUDA;
+    if (result_host &&
+        cudaMemcpyAsync(result_host, result_dev, sizeof(adloco_test_result), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return ADLOCO_ERR_CUDA;
+    return ADLOCO_OK;
+}
+
+namespace adloco {
+
+// ---------------------------------------------------------------------------------
 // outer step: K-way pseudo-gradient average + momentum update, one pass
 // ---------------------------------------------------------------------------------
 struct OuterArgs {
