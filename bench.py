@@ -179,6 +179,10 @@ def run_reference(args, rank):
 
 
 def workload_config():
+    if NT_P != 1 << 24:
+        return {"workload": f"profiling case: norm test B={NT_B} P={NT_P}, outer step K={OUT_K} P={OUT_P}, "
+                            f"Gram layer B={GR_B}", "l2": "inputs larger than L2 except the Gram layer",
+                "parallelism": "replicas"}
     return {"workload": "configs[1] streaming scale-up: norm test B=64 P=16,777,216 fp32 (eta 0.1/0.5/1.0) + "
                         "outer step K=8 bf16 P=124,439,808 (fp32 theta and momentum, lr 0.7, Nesterov 0.9); "
                         "plus configs[2] Gram layer B=32 T=1024 768->3072 bf16 for the tensor-core figure",
@@ -271,6 +275,21 @@ def run_ours(args, rank, world, local_rank):
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
     total_ms, stream_ms, gram_ms, nt_ms, os_ms = times.tolist()
 
+    # the two tensor-core kernels one by one (outside the timed steps): the call without a
+    # sum buffer runs the Gram kernel alone, the difference to the full call is the GEMM
+    reps = 20
+    g0, g1, g2 = ev(), ev(), ev()
+    g0.record(stream)
+    for _ in range(reps):
+        ctx.gram_sqnorm(X, D, n_layer)
+    g1.record(stream)
+    for _ in range(reps):
+        ctx.gram_sqnorm(X, D, n_layer, grad_sum=S_layer, accumulate_sum=True)
+    g2.record(stream)
+    torch.cuda.synchronize()
+    gram_only_ms = g0.elapsed_time(g1) / reps
+    mean_grad_ms = max(g1.elapsed_time(g2) / reps - gram_only_ms, 1e-6)
+
     nt_bytes, os_bytes = algorithmic_bytes()
     peaks = load_peaks()
     value = world * (nt_bytes + os_bytes) / (stream_ms * 1e-3) / 1e9
@@ -328,6 +347,16 @@ def run_ours(args, rank, world, local_rank):
                           "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                           "frac": (sym + mg) / (gram_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                           "algorithmic_flops": sym + mg, "includes": "gram + mean-grad + accumulate + finalize"},
+            "gram_sqnorm_kernel": {"bound": "tensor", "ms_per_launch": gram_only_ms,
+                                   "achieved": sym / (gram_only_ms * 1e-3) / 1e12,
+                                   "executed_tflops": executed / (gram_only_ms * 1e-3) / 1e12,
+                                   "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                   "frac": sym / (gram_only_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                   "algorithmic_flops": sym, "timed": "alone, back to back, incl. the memset of n"},
+            "mean_grad_kernel": {"bound": "tensor", "ms_per_launch": mean_grad_ms,
+                                 "achieved": mg / (mean_grad_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
+                                 "unit": "TFLOP/s", "frac": mg / (mean_grad_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                 "algorithmic_flops": mg, "timed": "full call minus the Gram-only call"},
         },
         "last_result": {"stat": last.stat, "b_req": last.b_req, "flags": last.flags},
     }
@@ -347,7 +376,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--small", action="store_true",
+                    help="profiling case: same kernels on inputs of a few hundred MB (not a bench value)")
     args = ap.parse_args()
+    if args.small:
+        global NT_P, OUT_P, GR_B
+        NT_P, OUT_P, GR_B = 1 << 21, 1 << 24, 8
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -40,42 +40,64 @@ __device__ __forceinline__ float warp_sum_f(float v) {
 // =====================================================================================
 // Gram kernel
 // =====================================================================================
-constexpr int GR_TILE = 128;                       // tokens per tile side (M = N = 128)
+// Work item = (sample i, 128-token row tile ti, one or two adjacent 128-token column
+// blocks c0, c0+1) on or above the diagonal of the T x T Gram matrices.  Row ti's
+// blocks ti..nt-1 are grouped in pairs from the diagonal outwards, a left-over
+// single block last; a pair is one 128x256 MMA tile (each operand byte fetched
+// into shared memory then feeds twice the math of a 128x128 tile, which is what
+// the L2 -> shared-memory path needs to keep the tensor pipe busy).
+constexpr int GR_TILE = 128;                       // tokens per block side
 constexpr int GR_BK = 64;                          // features per stage: 64 bf16 = one 128-byte swizzle row
-constexpr int GR_STAGES = 6;
-constexpr int GR_TILE_BYTES = GR_TILE * GR_BK * 2; // 16 KB
-constexpr int GR_STAGE_BYTES = 2 * GR_TILE_BYTES;  // t-tile and s-tile
+constexpr int GR_STAGES = 4;
+constexpr int GR_BLOCK_BYTES = GR_TILE * GR_BK * 2;          // 16 KB: 128 rows of one stage
+constexpr int GR_STAGE_BYTES = 3 * GR_BLOCK_BYTES;           // row tile + up to two column blocks
 constexpr int GR_SMEM = GR_STAGES * GR_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int GR_THREADS = 320;                              // warp 0 TMA, warp 1 MMA, warps 2-9 epilogue
 
 struct GramArgs {
     int B, T, d_in, d_out;
-    int nt;           // token tiles per sample
-    int pairs;        // nt (nt + 1) / 2 tile pairs (s >= t)
-    int total_items;  // B * pairs
-    float* n;         // [B], += (zeroed by the launcher unless accumulating)
+    int nt;               // 128-token blocks per sample side
+    int full_per_sample;  // items with two column blocks
+    int half_per_sample;  // items with one
+    int n_full;           // B * full_per_sample; items [0, n_full) are the two-block ones
+    int total_items;
+    float* n;             // [B], += (zeroed by the launcher unless accumulating)
     int* status;
 };
 
-__device__ __forceinline__ void gram_decode(int item, const GramArgs& a, int& i, int& ti, int& tj) {
-    i = item / a.pairs;
-    int p = item - i * a.pairs;
-    ti = 0;
-    while (p >= a.nt - ti) { p -= a.nt - ti; ++ti; }
-    tj = ti + p;
+__device__ __forceinline__ void gram_decode(int item, const GramArgs& a, int& i, int& ti, int& c0, int& ncb) {
+    const bool full = item < a.n_full;
+    int local;
+    if (full) {
+        i = item / a.full_per_sample;
+        local = item - i * a.full_per_sample;
+    } else {
+        const int h = item - a.n_full;
+        i = h / a.half_per_sample;
+        local = h - i * a.half_per_sample;
+    }
+    for (ti = 0; ti < a.nt - 1; ++ti) {
+        const int blocks = a.nt - ti;
+        const int cnt = full ? (blocks >> 1) : (blocks & 1);
+        if (local < cnt) break;
+        local -= cnt;
+    }
+    if (full) { c0 = ti + 2 * local; ncb = 2; }
+    else { c0 = a.nt - 1; ncb = 1; }
 }
 
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(GR_THREADS, 1)
 gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
                    const GramArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar_base = smem_base + GR_STAGES * GR_STAGE_BYTES;
-    // barrier slots (8 bytes each): full[S], empty[S], tmem_full[2], tmem_empty[2], drain
+    // barrier slots (8 bytes each): full[S], empty[S], tmem_full, tmem_empty, drain
     auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
     auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (GR_STAGES + s); };
-    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * GR_STAGES + b); };
-    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * GR_STAGES + 2 + b); };
-    const uint32_t drain_bar = bar_base + 8u * (2 * GR_STAGES + 4);
+    const uint32_t tfull_bar = bar_base + 8u * (2 * GR_STAGES);
+    const uint32_t tempty_bar = bar_base + 8u * (2 * GR_STAGES + 1);
+    const uint32_t drain_bar = bar_base + 8u * (2 * GR_STAGES + 2);
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -83,13 +105,14 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (uint32_t s = 0; s < GR_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        mbar_init(tfull_bar, 1);
+        mbar_init(tempty_bar, 8);
         mbar_init(drain_bar, 1);
         fence_barrier_init();
         prefetch_tmap(&tmX);
         prefetch_tmap(&tmD);
     }
-    if (warp == 1) {  // TMEM: two buffers of (X X^T | D D^T) accumulators, 128 columns each
+    if (warp == 1) {  // TMEM: X X^T accumulator in columns 0-255, D D^T in 256-511
         tmem_alloc(smem_u32(&tmem_base_slot), 512);
         tmem_relinquish();
     }
@@ -109,18 +132,19 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             uint32_t issued = 0;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < a.total_items; item += gridDim.x) {
-                int i, ti, tj;
-                gram_decode(item, a, i, ti, tj);
-                const bool diag = (ti == tj);
+                int i, ti, c0, ncb;
+                gram_decode(item, a, i, ti, c0, ncb);
                 for (int c = 0; c < chunks; ++c) {
                     if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
                     const bool is_x = c < kx;
                     const CUtensorMap* map = is_x ? &tmX : &tmD;
                     const int k0 = (is_x ? c : c - kx) * GR_BK;
                     const uint32_t sA = smem_base + ps.stage * GR_STAGE_BYTES;
-                    mbar_arrive_expect_tx(full_bar(ps.stage), diag ? GR_TILE_BYTES : GR_STAGE_BYTES);
+                    mbar_arrive_expect_tx(full_bar(ps.stage), (1 + ncb) * GR_BLOCK_BYTES);
                     tma_load_3d(sA, map, full_bar(ps.stage), k0, ti * GR_TILE, i);
-                    if (!diag) tma_load_3d(sA + GR_TILE_BYTES, map, full_bar(ps.stage), k0, tj * GR_TILE, i);
+                    tma_load_3d(sA + GR_BLOCK_BYTES, map, full_bar(ps.stage), k0, c0 * GR_TILE, i);
+                    if (ncb == 2)
+                        tma_load_3d(sA + 2 * GR_BLOCK_BYTES, map, full_bar(ps.stage), k0, (c0 + 1) * GR_TILE, i);
                     ++issued;
                     ps.advance(GR_STAGES);
                 }
@@ -139,24 +163,23 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16_f32(GR_TILE, GR_TILE, 0, 0);
             PipeState ps;
             bool ok = true;
             int n_item = 0;
             for (int item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++n_item) {
-                int i, ti, tj;
-                gram_decode(item, a, i, ti, tj);
-                const bool diag = (ti == tj);
-                const uint32_t buf = n_item & 1, use = n_item >> 1;
-                if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                int i, ti, c0, ncb;
+                gram_decode(item, a, i, ti, c0, ncb);
+                const uint32_t idesc = idesc_bf16_f32(GR_TILE, GR_TILE * ncb, 0, 0);
+                // the single accumulator pair must have been drained by the epilogue
+                if (!mbar_wait(tempty_bar, (n_item & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
                 tc_fence_after();
                 for (int c = 0; c < chunks; ++c) {
                     if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, kWaitLimitNs)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t acc = tmem_base + buf * 256u + (c < kx ? 0u : 128u);
+                    const uint32_t acc = tmem_base + (c < kx ? 0u : 256u);
                     const bool first = (c == 0 || c == kx);
                     const uint32_t sA = smem_base + ps.stage * GR_STAGE_BYTES;
-                    const uint32_t sB = diag ? sA : sA + GR_TILE_BYTES;
+                    const uint32_t sB = sA + GR_BLOCK_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < GR_BK / 16; ++kk) {
                         // K-major, 128-byte swizzle: rows of 128 B, 8-row groups 1024 B apart;
@@ -168,7 +191,7 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     mma_commit(empty_bar(ps.stage));   // stage reusable once these MMAs have read it
                     ps.advance(GR_STAGES);
                 }
-                if (ok) mma_commit(tfull_bar(buf));    // both accumulators of this item complete
+                if (ok) mma_commit(tfull_bar);         // both accumulators of this item complete
             }
             if (!ok) {
                 mma_commit(drain_bar);
@@ -178,31 +201,35 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         }
     } else {
         // ---------------- epilogue: sum over the tile of (X X^T) .* (D D^T) ----------------
-        const uint32_t q = warp & 3;   // TMEM lanes 32q .. 32q+31 belong to this warp
+        const uint32_t q = warp & 3;            // TMEM lanes 32q .. 32q+31 belong to this warp
+        const uint32_t half = (warp - 2) >> 2;  // which half of the tile's columns
         int n_item = 0;
         for (int item = blockIdx.x; item < a.total_items; item += gridDim.x, ++n_item) {
-            int i, ti, tj;
-            gram_decode(item, a, i, ti, tj);
-            const uint32_t buf = n_item & 1, use = n_item >> 1;
-            if (!mbar_wait(tfull_bar(buf), use & 1u, abortp, kWaitLimitNs)) break;
+            int i, ti, c0, ncb;
+            gram_decode(item, a, i, ti, c0, ncb);
+            if (!mbar_wait(tfull_bar, n_item & 1u, abortp, kWaitLimitNs)) break;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + buf * 256u;
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16);
+            const int cols_per_half = 64 * ncb;
+            const int col_begin = (int)half * cols_per_half;
             float sum = 0.f;
 #pragma unroll 1
-            for (int cc = 0; cc < GR_TILE / 32; ++cc) {
+            for (int col = col_begin; col < col_begin + cols_per_half; col += 32) {
                 uint32_t x[32], d[32];
-                tmem_ld32(taddr + cc * 32, x);
-                tmem_ld32(taddr + 128 + cc * 32, d);
+                tmem_ld32(taddr + col, x);
+                tmem_ld32(taddr + 256 + col, d);
                 tmem_ld_wait();
+                float part = 0.f;
 #pragma unroll
-                for (int e = 0; e < 32; ++e) sum = fmaf(__uint_as_float(x[e]), __uint_as_float(d[e]), sum);
+                for (int e = 0; e < 32; ++e) part = fmaf(__uint_as_float(x[e]), __uint_as_float(d[e]), part);
+                // blocks below the diagonal are never computed: an off-diagonal block counts twice
+                sum += (c0 + (col >> 7) == ti) ? part : 2.0f * part;
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            if (lane == 0) mbar_arrive(tempty_bar);
             const float w = warp_sum_f(sum);
-            // tiles below the diagonal are never computed: an off-diagonal tile counts twice
-            if (lane == 0) atomicAdd(a.n + i, ti == tj ? w : 2.0f * w);
+            if (lane == 0) atomicAdd(a.n + i, w);
         }
     }
 
@@ -460,10 +487,14 @@ int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     GramArgs a;
     a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
     a.nt = (int)((T + GR_TILE - 1) / GR_TILE);
-    const int64_t pairs = (int64_t)a.nt * (a.nt + 1) / 2;
-    if (pairs * B > 0x7fffffff) return ADLOCO_ERR_UNSUPPORTED;
-    a.pairs = (int)pairs;
-    a.total_items = (int)(pairs * B);
+    int64_t fulls = 0;
+    for (int ti = 0; ti < a.nt; ++ti) fulls += (a.nt - ti) / 2;
+    const int64_t halves = (a.nt + 1) / 2;
+    if ((fulls + halves) * B > 0x7fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    a.full_per_sample = (int)fulls;
+    a.half_per_sample = (int)halves;
+    a.n_full = (int)(fulls * B);
+    a.total_items = (int)((fulls + halves) * B);
     a.n = n; a.status = ctx->gemm_status;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
     static bool attr_set = false;
@@ -472,7 +503,7 @@ int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
         attr_set = true;
     }
     const int grid = a.total_items < ctx->sm_count ? a.total_items : ctx->sm_count;
-    gram_sqnorm_kernel<<<grid, TC_THREADS, GR_SMEM, st>>>(tmX, tmD, a);
+    gram_sqnorm_kernel<<<grid, GR_THREADS, GR_SMEM, st>>>(tmX, tmD, a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;

@@ -550,59 +550,62 @@ __device__ __forceinline__ void outer_update(float th, float v, double acc, cons
     th_new = (float)fma(-(double)a.lr, u, (double)th);
 }
 
+// Every thread owns four consecutive elements per iteration: theta and v arrive as
+// one 128-bit load each, an instance as 128 bits (fp32) or 64 bits (bf16), so all
+// accesses of a warp are contiguous and every fetched sector is used in full.
+template <bool BF16>
+__device__ __forceinline__ void load_inst4(const void* base, int64_t i, float (&x)[4]) {
+    if constexpr (BF16) {
+        const uint2 w = __ldcs(reinterpret_cast<const uint2*>(base) + i);
+        x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
+    } else {
+        const float4 w = __ldcs(reinterpret_cast<const float4*>(base) + i);
+        x[0] = w.x; x[1] = w.y; x[2] = w.z; x[3] = w.w;
+    }
+}
+
 template <bool BF16, bool WB>
-__global__ void __launch_bounds__(256) outer_step_kernel(const __grid_constant__ OuterArgs a) {
-    constexpr int VEC = BF16 ? 8 : 4;
+__global__ void __launch_bounds__(256, 6) outer_step_kernel(const __grid_constant__ OuterArgs a) {
+    constexpr int VEC = 4;
+    constexpr int KB = 4;   // instance loads issued back to back
     const int64_t nvec = a.P / VEC;
     const int64_t step = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
-        float th[VEC], v[VEC];
+        const float4 t4 = __ldcs(reinterpret_cast<const float4*>(a.th_in) + i);
+        const float4 v4 = __ldcs(reinterpret_cast<const float4*>(a.v_in) + i);
+        const float th[VEC] = {t4.x, t4.y, t4.z, t4.w};
+        const float v[VEC] = {v4.x, v4.y, v4.z, v4.w};
         double acc[VEC], thd[VEC];
-        {
-            const float4* tp = reinterpret_cast<const float4*>(a.th_in) + i * (VEC / 4);
-            const float4* vp = reinterpret_cast<const float4*>(a.v_in) + i * (VEC / 4);
-#pragma unroll
-            for (int h = 0; h < VEC / 4; ++h) {
-                const float4 t = __ldcs(tp + h), w = __ldcs(vp + h);
-                th[4 * h] = t.x; th[4 * h + 1] = t.y; th[4 * h + 2] = t.z; th[4 * h + 3] = t.w;
-                v[4 * h] = w.x; v[4 * h + 1] = w.y; v[4 * h + 2] = w.z; v[4 * h + 3] = w.w;
-            }
-        }
 #pragma unroll
         for (int e = 0; e < VEC; ++e) { acc[e] = 0.0; thd[e] = (double)th[e]; }
-#pragma unroll 4
-        for (int k = 0; k < a.K; ++k) {
-            if (BF16) {
-                const uint4 x = __ldcs(reinterpret_cast<const uint4*>(a.inst[k]) + i);
-                acc[0] += thd[0] - (double)bf16_lo(x.x); acc[1] += thd[1] - (double)bf16_hi(x.x);
-                acc[2] += thd[2] - (double)bf16_lo(x.y); acc[3] += thd[3] - (double)bf16_hi(x.y);
-                acc[4 % VEC] += thd[4 % VEC] - (double)bf16_lo(x.z); acc[5 % VEC] += thd[5 % VEC] - (double)bf16_hi(x.z);
-                acc[6 % VEC] += thd[6 % VEC] - (double)bf16_lo(x.w); acc[7 % VEC] += thd[7 % VEC] - (double)bf16_hi(x.w);
-            } else {
-                const float4 x = __ldcs(reinterpret_cast<const float4*>(a.inst[k]) + i);
-                acc[0] += thd[0] - (double)x.x; acc[1] += thd[1] - (double)x.y; acc[2] += thd[2] - (double)x.z; acc[3] += thd[3] - (double)x.w;
-            }
+        int k = 0;
+        for (; k + KB <= a.K; k += KB) {
+            float x[KB][VEC];
+#pragma unroll
+            for (int u = 0; u < KB; ++u) load_inst4<BF16>(a.inst[k + u], i, x[u]);
+#pragma unroll
+            for (int u = 0; u < KB; ++u)
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[e] += thd[e] - (double)x[u][e];
+        }
+        for (; k < a.K; ++k) {
+            float x[VEC];
+            load_inst4<BF16>(a.inst[k], i, x);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] += thd[e] - (double)x[e];
         }
         float tn[VEC], vn[VEC];
 #pragma unroll
         for (int e = 0; e < VEC; ++e) outer_update(th[e], v[e], acc[e], a, tn[e], vn[e]);
-        float4* to = reinterpret_cast<float4*>(a.th_out) + i * (VEC / 4);
-        float4* vo = reinterpret_cast<float4*>(a.v_out) + i * (VEC / 4);
-#pragma unroll
-        for (int h = 0; h < VEC / 4; ++h) {
-            __stcs(to + h, make_float4(tn[4 * h], tn[4 * h + 1], tn[4 * h + 2], tn[4 * h + 3]));
-            __stcs(vo + h, make_float4(vn[4 * h], vn[4 * h + 1], vn[4 * h + 2], vn[4 * h + 3]));
-        }
+        __stcs(reinterpret_cast<float4*>(a.th_out) + i, make_float4(tn[0], tn[1], tn[2], tn[3]));
+        __stcs(reinterpret_cast<float4*>(a.v_out) + i, make_float4(vn[0], vn[1], vn[2], vn[3]));
         if (WB) {
-            for (int k = 0; k < a.K; ++k) {
-                if (a.wb[k] == nullptr) continue;
+            for (int kk = 0; kk < a.K; ++kk) {
+                if (a.wb[kk] == nullptr) continue;
                 if (BF16) {
-                    uint4 o;
-                    o.x = pack_bf16(tn[0], tn[1]); o.y = pack_bf16(tn[2], tn[3]);
-                    o.z = pack_bf16(tn[4 % VEC], tn[5 % VEC]); o.w = pack_bf16(tn[6 % VEC], tn[7 % VEC]);
-                    reinterpret_cast<uint4*>(a.wb[k])[i] = o;
+                    reinterpret_cast<uint2*>(a.wb[kk])[i] = make_uint2(pack_bf16(tn[0], tn[1]), pack_bf16(tn[2], tn[3]));
                 } else {
-                    reinterpret_cast<float4*>(a.wb[k])[i] = make_float4(tn[0], tn[1], tn[2], tn[3]);
+                    reinterpret_cast<float4*>(a.wb[kk])[i] = make_float4(tn[0], tn[1], tn[2], tn[3]);
                 }
             }
         }
@@ -633,9 +636,14 @@ __global__ void __launch_bounds__(256) outer_step_kernel(const __grid_constant__
     }
 }
 
-static unsigned elementwise_grid(const adloco_ctx* ctx, int64_t nvec, int threads, int blocks_per_sm) {
+// Persistent grid for the elementwise kernels: as many blocks as are resident at
+// once (so no partial last wave), fewer when the problem is smaller than that.
+template <typename Kern>
+static unsigned elementwise_grid(const adloco_ctx* ctx, Kern kern, int64_t nvec, int threads) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
     int64_t want = (nvec + threads - 1) / threads;
-    const int64_t cap = (int64_t)ctx->sm_count * blocks_per_sm;
+    const int64_t cap = (int64_t)ctx->sm_count * per_sm;
     if (want > cap) want = cap;
     if (want < 1) want = 1;
     return (unsigned)want;
@@ -649,14 +657,13 @@ int launch_outer_step(adloco_ctx* ctx, const OuterLaunch& l, cudaStream_t st) {
     }
     a.th_in = l.th_in; a.th_out = l.th_out; a.v_in = l.v_in; a.v_out = l.v_out;
     a.P = l.P; a.lr = l.lr; a.mu = l.mu; a.invK = 1.0 / (double)l.K; a.K = l.K; a.nesterov = l.nesterov;
-    const int vec = l.bf16 ? 8 : 4;
-    const unsigned grid = elementwise_grid(ctx, l.P / vec, 256, 8);
+    const int64_t nvec = l.P / 4;
     if (l.bf16) {
-        if (l.has_wb) outer_step_kernel<true, true><<<grid, 256, 0, st>>>(a);
-        else outer_step_kernel<true, false><<<grid, 256, 0, st>>>(a);
+        if (l.has_wb) outer_step_kernel<true, true><<<elementwise_grid(ctx, outer_step_kernel<true, true>, nvec, 256), 256, 0, st>>>(a);
+        else outer_step_kernel<true, false><<<elementwise_grid(ctx, outer_step_kernel<true, false>, nvec, 256), 256, 0, st>>>(a);
     } else {
-        if (l.has_wb) outer_step_kernel<false, true><<<grid, 256, 0, st>>>(a);
-        else outer_step_kernel<false, false><<<grid, 256, 0, st>>>(a);
+        if (l.has_wb) outer_step_kernel<false, true><<<elementwise_grid(ctx, outer_step_kernel<false, true>, nvec, 256), 256, 0, st>>>(a);
+        else outer_step_kernel<false, false><<<elementwise_grid(ctx, outer_step_kernel<false, false>, nvec, 256), 256, 0, st>>>(a);
     }
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
@@ -730,9 +737,8 @@ int launch_merge(adloco_ctx* ctx, const MergeLaunch& l, cudaStream_t st) {
     }
     a.out = l.out; a.P = l.P; a.K = l.K;
     const int vec = l.bf16 ? 8 : 4;
-    const unsigned grid = elementwise_grid(ctx, l.P / vec, 256, 8);
-    if (l.bf16) merge_kernel<true><<<grid, 256, 0, st>>>(a);
-    else merge_kernel<false><<<grid, 256, 0, st>>>(a);
+    if (l.bf16) merge_kernel<true><<<elementwise_grid(ctx, merge_kernel<true>, l.P / vec, 256), 256, 0, st>>>(a);
+    else merge_kernel<false><<<elementwise_grid(ctx, merge_kernel<false>, l.P / vec, 256), 256, 0, st>>>(a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;

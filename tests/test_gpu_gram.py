@@ -69,12 +69,13 @@ def test_accumulate_flags_and_unsupported_shapes(ctx):
     n2, S2 = n.clone(), S.clone()
     ctx.gram_sqnorm(X, D, n2, accumulate_norms=True, grad_sum=S2, accumulate_sum=True)
     torch.cuda.synchronize()
-    assert torch.allclose(n2, 2 * n, rtol=1e-6) and torch.allclose(S2, 2 * S, rtol=1e-6, atol=1e-9)
+    # fp32 reductions into S arrive in no fixed order: allow for a few ulp of the largest terms
+    assert torch.allclose(n2, 2 * n, rtol=1e-5) and torch.allclose(S2, 2 * S, rtol=1e-5, atol=1e-5 * float(S.abs().max()))
     # without the sum buffer only the norms are computed
     n3 = torch.zeros(2, device=DEV)
     ctx.gram_sqnorm(X, D, n3)
     torch.cuda.synchronize()
-    assert torch.equal(n3, n)
+    assert torch.allclose(n3, n, rtol=1e-5)
     Xb, Db = W.linear_layer(2, 16, 12, 64, seed=1, device=DEV)      # d_in not a multiple of 8
     before = ctx.launch_count
     with pytest.raises(A.AdlocoError) as e:
