@@ -2,7 +2,7 @@
 //
 //   gram_sqnorm_kernel  n_i = <X_i X_i^T, D_i D_i^T>_F, the squared Frobenius norm of
 //                       sample i's weight gradient D_i^T X_i, without forming it:
-//                       for every 128x128 tile (t, s >= t) of the token-by-token
+//                       for every tile on or above the diagonal of the token-by-token
 //                       Gram matrices both products are accumulated in TMEM and the
 //                       epilogue reduces their elementwise product.
 //   mean_grad_kernel    S (+)= sum_i D_i^T X_i, the batch gradient sum, a GEMM whose
@@ -10,9 +10,9 @@
 //
 // Both are persistent, warp-specialised kernels: warp 0 issues TMA tile loads
 // into a ring of shared-memory stages, warp 1 issues tcgen05.mma from shared
-// memory into TMEM accumulators (double-buffered), warps 2-5 drain the
-// accumulators.  Every wait is bounded; a wait that runs out raises a status
-// word and all roles leave through the common teardown.
+// memory into TMEM accumulators, the remaining warps drain the accumulators.
+// Every wait is bounded; a wait that runs out raises a status word and all
+// roles leave through the common teardown.
 #include "common.cuh"
 #include "ptx.cuh"
 
