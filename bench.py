@@ -61,6 +61,27 @@ def gram_flops():
     return sym, executed, mean_grad
 
 
+def reduce_max_over_ranks(values, device="cpu"):
+    """Max over ranks of each entry (the time of a multi-rank step is its slowest
+    rank's); identity when no process group is initialised."""
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_throughput(units_per_rank: float, world: int, max_seconds: float) -> float:
+    """Whole-job throughput of `world` replicas that each process `units_per_rank`."""
+    return world * units_per_rank / max_seconds
+
+
+# DRAM traffic of norm_test_kernel per gradient element, from the ncu capture of the
+# profiling case (B=64, P=2^21: 536.98 MB read + 4.28 MB written for 2^27 elements);
+# traffic grows in proportion to B*P, so a full launch is this times its element count.
+NT_TRAFFIC_BYTES_PER_ELEMENT = (536.978e6 + 4.280e6) / float(64 * (1 << 21))
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -129,7 +150,7 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------
 def oracle_sample_run(steps: int, warmup: int):
     """Times the oracle, as it stands, on a bounded sample of the streaming
-    workload: the norm test on B=64 x P=2^19 and the outer step on K=8 x P=2^21.
+    workload: the norm test on B=64 x P=2^22 and the outer step on K=8 x P=2^23.
     Returns (GB/s over the sample's algorithmic bytes, ms per step, threads)."""
     import numpy as np
     import oracle.adloco_oracle as O
@@ -138,7 +159,7 @@ def oracle_sample_run(steps: int, warmup: int):
         threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
         threads = 1
-    sP, oP = 1 << 19, 1 << 21
+    sP, oP = 1 << 22, 1 << 23
     G = W.to_numpy(W.per_sample_grads(NT_B, sP, sigma=0.5, seed=1))
     theta, inst, mom = W.outer_state(OUT_K, oP, inst_dtype=torch.bfloat16, seed=2)
     th, v, ins = W.to_numpy(theta), W.to_numpy(mom), [W.to_numpy(t) for t in inst]
@@ -156,7 +177,7 @@ def oracle_sample_run(steps: int, warmup: int):
     for _ in range(steps):
         one()
     dt = (time.perf_counter() - t0) / max(steps, 1)
-    sample = f"norm test B={NT_B} P=2^19 fp32 + outer step K={OUT_K} bf16 P=2^21 (1/32 resp. 1/59 of the workload)"
+    sample = f"norm test B={NT_B} P=2^22 fp32 + outer step K={OUT_K} bf16 P=2^23 (1/4 resp. 1/15 of the workload)"
     return nbytes / dt / 1e9, dt * 1e3, threads, sample
 
 
@@ -269,11 +290,8 @@ def run_ours(args, rank, world, local_rank):
     os_ms = sum(m["os0"].elapsed_time(m["os1"]) for m in marks) / args.steps
     stream_ms = sum(m["nt0"].elapsed_time(m["os1"]) for m in marks) / args.steps
     gram_ms = sum(m["os1"].elapsed_time(m["gr1"]) for m in marks) / args.steps
-    times = torch.tensor([total_ms, stream_ms, gram_ms, nt_ms, os_ms], dtype=torch.float64, device=dev)
-    if use_dist:
-        import torch.distributed as dist
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, stream_ms, gram_ms, nt_ms, os_ms = times.tolist()
+    total_ms, stream_ms, gram_ms, nt_ms, os_ms = reduce_max_over_ranks(
+        [total_ms, stream_ms, gram_ms, nt_ms, os_ms], device=dev)
 
     # the two tensor-core kernels one by one (outside the timed steps): the call without a
     # sum buffer runs the Gram kernel alone, the difference to the full call is the GEMM
@@ -292,7 +310,7 @@ def run_ours(args, rank, world, local_rank):
 
     nt_bytes, os_bytes = algorithmic_bytes()
     peaks = load_peaks()
-    value = world * (nt_bytes + os_bytes) / (stream_ms * 1e-3) / 1e9
+    value = aggregate_throughput(nt_bytes + os_bytes, world, stream_ms * 1e-3) / 1e9
     sym, executed, mg = gram_flops()
 
     # ---- end to end through the host-memory entry points (rank-local pinned buffers)
@@ -314,12 +332,10 @@ def run_ours(args, rank, world, local_rank):
                 pass                                        # the eta sweep needs no further data movement
             ctx.outer_step_host(inst_h, th_h, v_h, lr=LR, momentum=MU)
         torch.cuda.synchronize()
-        e2e_s = torch.tensor([(time.perf_counter() - t0) / reps], dtype=torch.float64, device=dev)
-        if use_dist:
-            dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * (nt_bytes + os_bytes) / e2e_s.item() / 1e9, "unit": UNIT,
+        e2e_s = reduce_max_over_ranks([(time.perf_counter() - t0) / reps], device=dev)[0]
+        e2e = {"value": aggregate_throughput(nt_bytes + os_bytes, world, e2e_s) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": nt_bytes + (2 * OUT_K + 8) * OUT_P,
-               "d2h_bytes_per_step": 8 * OUT_P + 80, "ms_per_step": e2e_s.item() * 1e3, "steps": reps}
+               "d2h_bytes_per_step": 8 * OUT_P + 80, "ms_per_step": e2e_s * 1e3, "steps": reps}
         del Gh, th_h, v_h, inst_h
 
     if rank != 0:
@@ -335,7 +351,8 @@ def run_ours(args, rank, world, local_rank):
         "gpu_launches": launches,
         "stream_ms_per_step": stream_ms,
         "roofline": {"bound": "hbm", "kernel": "norm_test_kernel", "achieved": nt_gbs, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": nt_gbs / peaks["hbm_gbs"], "traffic": None,
+                     "unit": "GB/s", "frac": nt_gbs / peaks["hbm_gbs"],
+                     "traffic": NT_TRAFFIC_BYTES_PER_ELEMENT * NT_B * NT_P,
                      "peak_source": peaks["source"], "ms_per_launch": nt_ms, "algorithmic_bytes": nt_bytes},
         "kernels": {
             "outer_step_kernel": {"bound": "hbm", "achieved": os_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
