@@ -22,7 +22,6 @@ using namespace ptx;
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
 constexpr uint64_t kDrainLimitNs = 50000000ull;    // 50 ms per barrier while leaving after a time-out
-constexpr int TC_THREADS = 192;
 
 struct PipeState {
     uint32_t stage = 0, phase = 0;
@@ -134,14 +133,16 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             for (int item = blockIdx.x; ok && item < a.total_items; item += gridDim.x) {
                 int i, ti, c0, ncb;
                 gram_decode(item, a, i, ti, c0, ncb);
+                // on the diagonal the row tile is the first column block: fetch it once
+                const bool diag = (c0 == ti);
                 for (int c = 0; c < chunks; ++c) {
                     if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
                     const bool is_x = c < kx;
                     const CUtensorMap* map = is_x ? &tmX : &tmD;
                     const int k0 = (is_x ? c : c - kx) * GR_BK;
                     const uint32_t sA = smem_base + ps.stage * GR_STAGE_BYTES;
-                    mbar_arrive_expect_tx(full_bar(ps.stage), (1 + ncb) * GR_BLOCK_BYTES);
-                    tma_load_3d(sA, map, full_bar(ps.stage), k0, ti * GR_TILE, i);
+                    mbar_arrive_expect_tx(full_bar(ps.stage), ((diag ? 0 : 1) + ncb) * GR_BLOCK_BYTES);
+                    if (!diag) tma_load_3d(sA, map, full_bar(ps.stage), k0, ti * GR_TILE, i);
                     tma_load_3d(sA + GR_BLOCK_BYTES, map, full_bar(ps.stage), k0, c0 * GR_TILE, i);
                     if (ncb == 2)
                         tma_load_3d(sA + 2 * GR_BLOCK_BYTES, map, full_bar(ps.stage), k0, (c0 + 1) * GR_TILE, i);
@@ -178,8 +179,8 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     tc_fence_after();
                     const uint32_t acc = tmem_base + (c < kx ? 0u : 256u);
                     const bool first = (c == 0 || c == kx);
-                    const uint32_t sA = smem_base + ps.stage * GR_STAGE_BYTES;
-                    const uint32_t sB = sA + GR_BLOCK_BYTES;
+                    const uint32_t sB = smem_base + ps.stage * GR_STAGE_BYTES + GR_BLOCK_BYTES;
+                    const uint32_t sA = (c0 == ti) ? sB : sB - GR_BLOCK_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < GR_BK / 16; ++kk) {
                         // K-major, 128-byte swizzle: rows of 128 B, 8-row groups 1024 B apart;
@@ -246,15 +247,20 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 // =====================================================================================
 // mean-gradient kernel: S[d_out, d_in] += sum over samples and tokens of delta x^T
 // =====================================================================================
-constexpr int MG_BM = 128;                          // d_out rows per tile
+// Output tile 256 (d_out) x 256 (d_in): two M=128 MMAs per K step share the X
+// operand, their accumulators fill all 512 TMEM columns.  Per byte fetched into
+// shared memory this does 128 flops, which is what lets the tensor pipe run
+// ahead of the L2 -> shared-memory path (a 128x256 tile does 85).
+constexpr int MG_BM = 256;                          // d_out rows per tile (two MMA halves of 128)
 constexpr int MG_BN = 256;                          // d_in columns per tile
 constexpr int MG_BK = 64;                           // tokens per stage
-constexpr int MG_STAGES = 4;
+constexpr int MG_STAGES = 3;
 constexpr int MG_BOX_BYTES = 64 * MG_BK * 2;        // one TMA box: 64 features x 64 tokens = 8 KB
 constexpr int MG_A_BYTES = (MG_BM / 64) * MG_BOX_BYTES;
 constexpr int MG_B_BYTES = (MG_BN / 64) * MG_BOX_BYTES;
-constexpr int MG_STAGE_BYTES = MG_A_BYTES + MG_B_BYTES;   // 48 KB
+constexpr int MG_STAGE_BYTES = MG_A_BYTES + MG_B_BYTES;   // 64 KB
 constexpr int MG_SMEM = MG_STAGES * MG_STAGE_BYTES + 1024 + 256;
+constexpr int MG_THREADS = 320;                     // warp 0 TMA, warp 1 MMA, warps 2-9 epilogue
 
 struct MeanGradArgs {
     int B, T, d_in, d_out;
@@ -264,7 +270,7 @@ struct MeanGradArgs {
     int* status;
 };
 
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(MG_THREADS, 1)
 mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
                  const MeanGradArgs a) {
     extern __shared__ uint8_t smem_raw[];
@@ -272,9 +278,9 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     const uint32_t bar_base = smem_base + MG_STAGES * MG_STAGE_BYTES;
     auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
     auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (MG_STAGES + s); };
-    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * MG_STAGES + b); };
-    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * MG_STAGES + 2 + b); };
-    const uint32_t drain_bar = bar_base + 8u * (2 * MG_STAGES + 4);
+    const uint32_t tfull_bar = bar_base + 8u * (2 * MG_STAGES);
+    const uint32_t tempty_bar = bar_base + 8u * (2 * MG_STAGES + 1);
+    const uint32_t drain_bar = bar_base + 8u * (2 * MG_STAGES + 2);
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -282,14 +288,15 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (uint32_t s = 0; s < MG_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        mbar_init(tfull_bar, 1);
+        mbar_init(tempty_bar, 8);
         mbar_init(drain_bar, 1);
         fence_barrier_init();
         prefetch_tmap(&tmX);
         prefetch_tmap(&tmD);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&tmem_base_slot), 512);   // two 128x256 fp32 accumulators
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);   // rows 0-127 in columns 0-255, rows 128-255 in 256-511
         tmem_relinquish();
     }
     tc_fence_before();
@@ -339,7 +346,7 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     } else if (warp == 1) {
         if (lane == 0) {
             // both operands are stored with the contraction index (tokens) strided: MN-major
-            constexpr uint32_t idesc = idesc_bf16_f32(MG_BM, MG_BN, 1, 1);
+            constexpr uint32_t idesc = idesc_bf16_f32(128, MG_BN, 1, 1);
             PipeState ps;
             bool ok = true;
             int seg = 0;
@@ -348,10 +355,8 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                 const int tile = (int)(u / a.B);
                 int64_t u_end = (int64_t)(tile + 1) * a.B;     // end of this tile's samples
                 if (u_end > u1) u_end = u1;
-                const uint32_t buf = seg & 1, use = seg >> 1;
-                if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                if (!mbar_wait(tempty_bar, (seg & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t acc = tmem_base + buf * 256u;
                 bool first = true;
                 for (; ok && u < u_end; ++u) {
                     for (int c = 0; c < kt; ++c) {
@@ -364,16 +369,19 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                             // MN-major, 128-byte swizzle: a token is a 128-byte row of 64 features,
                             // 8-token groups 1024 B apart (stride offset), the next 64 features one
                             // box further (leading offset); 16 tokens = 2 KB per MMA
-                            const uint64_t da = smem_desc_sw128(sA + kk * 2048, MG_BOX_BYTES, 1024);
                             const uint64_t db = smem_desc_sw128(sB + kk * 2048, MG_BOX_BYTES, 1024);
-                            mma_bf16(acc, da, db, idesc, (first && kk == 0) ? 0u : 1u);
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const uint64_t da = smem_desc_sw128(sA + h * 2 * MG_BOX_BYTES + kk * 2048, MG_BOX_BYTES, 1024);
+                                mma_bf16(tmem_base + h * 256u, da, db, idesc, (first && kk == 0) ? 0u : 1u);
+                            }
                         }
                         first = false;
                         mma_commit(empty_bar(ps.stage));
                         ps.advance(MG_STAGES);
                     }
                 }
-                if (ok) mma_commit(tfull_bar(buf));
+                if (ok) mma_commit(tfull_bar);
                 ++seg;
             }
             if (!ok) {
@@ -383,7 +391,8 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             }
         }
     } else {
-        const uint32_t q = warp & 3;
+        const uint32_t q = warp & 3;            // TMEM lane quarter
+        const uint32_t half = (warp - 2) >> 2;  // rows 0-127 or 128-255 of the tile
         int seg = 0;
         int64_t u = u0;
         while (u < u1) {
@@ -391,11 +400,10 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             int64_t u_end = (int64_t)(tile + 1) * a.B;
             if (u_end > u1) u_end = u1;
             const int tm = tile / a.ntn, tn = tile % a.ntn;
-            const uint32_t buf = seg & 1, use = seg >> 1;
-            if (!mbar_wait(tfull_bar(buf), use & 1u, abortp, kWaitLimitNs)) break;
+            if (!mbar_wait(tfull_bar, seg & 1u, abortp, kWaitLimitNs)) break;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + buf * 256u;
-            const int m = tm * MG_BM + (int)q * 32 + lane;
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + half * 256u;
+            const int m = tm * MG_BM + (int)half * 128 + (int)q * 32 + lane;
             float* srow = a.S + (int64_t)m * a.d_in;
 #pragma unroll 1
             for (int cc = 0; cc < MG_BN / 32; ++cc) {
@@ -421,7 +429,7 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            if (lane == 0) mbar_arrive(tempty_bar);
             u = u_end;
             ++seg;
         }
@@ -530,7 +538,7 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
         attr_set = true;
     }
     const int grid = a.units < ctx->sm_count ? (int)a.units : ctx->sm_count;
-    mean_grad_kernel<<<grid, TC_THREADS, MG_SMEM, st>>>(tmX, tmD, a);
+    mean_grad_kernel<<<grid, MG_THREADS, MG_SMEM, st>>>(tmX, tmD, a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;
