@@ -189,6 +189,20 @@ int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
                        int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
                        int accumulate_sum, void* stream);
 
+/* Same outputs as adloco_gram_sqnorm (n_i and, optionally, S; same argument
+ * meaning and limits) with a choice of route:
+ *   ADLOCO_LINEAR_GRAM    the Gram identity (adloco_gram_sqnorm)
+ *   ADLOCO_LINEAR_DIRECT  each sample's gradient tile G_i = D_i^T X_i (Eq. 1 applied to
+ *                         W, before the mean) is formed in tensor memory, squared and
+ *                         summed into n_i and added into S on chip; G_i never reaches HBM.
+ *                         One GEMM of 2 B T d_in d_out flops gives both outputs.
+ *   ADLOCO_LINEAR_AUTO    whichever executes fewer tensor-core flops for the shape
+ *                         (direct wins when T exceeds about d_in d_out / (d_in + d_out)). */
+enum { ADLOCO_LINEAR_AUTO = 0, ADLOCO_LINEAR_GRAM = 1, ADLOCO_LINEAR_DIRECT = 2 };
+int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                         int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
+                         int accumulate_sum, int method, void* stream);
+
 /* ---- switch-mode accumulation -------------------------------------------- */
 
 /* Accumulator of the test sums over the micro-batches of one large batch:

@@ -22,7 +22,7 @@ FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN = 1, 2, 4, 8
 # every symbol that include/adloco.h declares
 EXPORTS = (
     "adloco_create", "adloco_destroy", "adloco_status_string", "adloco_last_cuda_error", "adloco_launch_count",
-    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_gram_sqnorm",
+    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_gram_sqnorm", "adloco_linear_sqnorm",
     "adloco_accum_create", "adloco_accum_reset", "adloco_accum_destroy", "adloco_accumulate",
     "adloco_accum_finalize", "adloco_outer_step", "adloco_outer_step_host", "adloco_check_merge", "adloco_merge",
 )
@@ -80,6 +80,7 @@ def load_library() -> C.CDLL:
         "adloco_norm_test_host": (C.c_int, [vp, vp, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp]),
         "adloco_norm_test_noalloc": (C.c_int, [vp, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp, vp]),
         "adloco_gram_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
+        "adloco_linear_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, C.c_int, vp]),
         "adloco_accum_create": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), i32]),
         "adloco_accum_reset": (C.c_int, [vp, vp, vp]),
         "adloco_accum_destroy": (C.c_int, [vp]),
@@ -211,6 +212,19 @@ class Context:
                                          int(accumulate_norms), _ptr(grad_sum), int(accumulate_sum),
                                          _stream(stream))
         self.check(rc, "adloco_gram_sqnorm")
+
+    def linear_sqnorm(self, X, D, per_sample_sqnorm, *, method="auto", accumulate_norms=False, grad_sum=None,
+                      accumulate_sum=False, stream=None):
+        """adloco_linear_sqnorm: method is "auto", "gram" or "direct"."""
+        B, T, d_in = X.shape
+        d_out = D.shape[2]
+        if X.dtype != torch.bfloat16 or D.dtype != torch.bfloat16 or not X.is_contiguous() or not D.is_contiguous():
+            raise AdlocoError(ERR_INVALID_ARG, "X and D must be contiguous bfloat16")
+        code = {"auto": 0, "gram": 1, "direct": 2}[method]
+        rc = self.lib.adloco_linear_sqnorm(self.h, _ptr(X), _ptr(D), B, T, d_in, d_out, _ptr(per_sample_sqnorm),
+                                           int(accumulate_norms), _ptr(grad_sum), int(accumulate_sum), code,
+                                           _stream(stream))
+        self.check(rc, "adloco_linear_sqnorm")
 
     # ------------------------------------------------------------------ outer step
     def outer_step(self, instances, theta_in, mom_in, *, lr, momentum, nesterov=True, theta_out=None,

@@ -241,6 +241,33 @@ int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     return rc;
 }
 
+int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                         int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
+                         int accumulate_sum, int method, void* stream) {
+    if (method != ADLOCO_LINEAR_AUTO && method != ADLOCO_LINEAR_GRAM && method != ADLOCO_LINEAR_DIRECT)
+        return ADLOCO_ERR_INVALID_ARG;
+    if (!ctx || !X || !D || !per_sample_sqnorm) return ADLOCO_ERR_INVALID_ARG;
+    if (B < 1 || T < 1 || d_in < 1 || d_out < 1) return ADLOCO_ERR_INVALID_ARG;
+    if (method == ADLOCO_LINEAR_AUTO) {
+        // tensor work of the two routes, at the granularity the kernels execute
+        const double nt = (double)((T + 127) / 128);
+        const double gram = 2.0 * (double)B * (nt * (nt + 1) / 2) * 128.0 * 128.0 * (double)(d_in + d_out) +
+                            (grad_sum ? 2.0 * (double)B * (double)T * (double)d_in * (double)d_out : 0.0);
+        const double direct = 2.0 * (double)B * (double)T * (double)d_in * (double)d_out;
+        method = direct <= gram ? ADLOCO_LINEAR_DIRECT : ADLOCO_LINEAR_GRAM;
+    }
+    if (method == ADLOCO_LINEAR_GRAM)
+        return adloco_gram_sqnorm(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, grad_sum,
+                                  accumulate_sum, stream);
+    if ((d_in % 8) != 0 || (d_out % 8) != 0) return ADLOCO_ERR_UNSUPPORTED;
+    if (B > (1 << 30) || T > (1 << 30) || d_in > (1 << 30) || d_out > (1 << 30)) return ADLOCO_ERR_UNSUPPORTED;
+    if (!aligned16(X) || !aligned16(D)) return ADLOCO_ERR_ALIGNMENT;
+    if (grad_sum && !aligned16(grad_sum)) return ADLOCO_ERR_ALIGNMENT;
+    DeviceGuard g(ctx->device);
+    return launch_direct_sqnorm(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, grad_sum,
+                                accumulate_sum, static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------------------------
 // switch-mode accumulator
 // ---------------------------------------------------------------------------------

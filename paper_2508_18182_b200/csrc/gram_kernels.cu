@@ -244,6 +244,32 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
 }
 
+// Work split shared by the two token-contraction kernels.  The (tile, sample) units of
+// one output tile are cut into `splits` chunks of `chunk` consecutive samples, every
+// chunk starting at a multiple of `chunk`; work item j = (tile j / splits, chunk
+// j % splits).  CTAs that start together therefore walk through the same few samples
+// at the same time, which keeps the operands of those samples resident in L2 (a plain
+// even split lets the CTAs drift over all samples and doubles the DRAM reads).
+struct SplitPlan {
+    int splits, chunk, items;
+};
+static SplitPlan make_split(int64_t tiles, int64_t B, int sm_count) {
+    SplitPlan p;
+    int64_t s = tiles >= sm_count ? 1 : sm_count / tiles;
+    if (s > B) s = B;
+    p.chunk = (int)((B + s - 1) / s);
+    p.splits = (int)((B + p.chunk - 1) / p.chunk);
+    p.items = (int)(tiles * p.splits);
+    return p;
+}
+__device__ __forceinline__ void item_range(int item, int splits, int chunk, int B, int64_t& u0, int64_t& u1) {
+    const int tile = item / splits, k = item - tile * splits;
+    const int b0 = k * chunk;
+    const int b1 = b0 + chunk < B ? b0 + chunk : B;
+    u0 = (int64_t)tile * B + b0;
+    u1 = (int64_t)tile * B + b1;
+}
+
 // =====================================================================================
 // mean-gradient kernel: S[d_out, d_in] += sum over samples and tokens of delta x^T
 // =====================================================================================
@@ -265,7 +291,7 @@ constexpr int MG_THREADS = 320;                     // warp 0 TMA, warp 1 MMA, w
 struct MeanGradArgs {
     int B, T, d_in, d_out;
     int ntm, ntn;       // tiles along d_out, d_in
-    int64_t units;      // ntm * ntn * B (tile-major, sample-minor)
+    int splits, chunk, items;   // see SplitPlan
     float* S;           // [d_out, d_in], += (zeroed by the launcher unless accumulating)
     int* status;
 };
@@ -305,9 +331,6 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
 
-    // this CTA's contiguous share of the (tile, sample) units
-    const int64_t u0 = a.units * blockIdx.x / gridDim.x;
-    const int64_t u1 = a.units * (blockIdx.x + 1) / gridDim.x;
     const int kt = (a.T + MG_BK - 1) / MG_BK;
 
     if (warp == 0) {
@@ -315,6 +338,9 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             PipeState ps;
             uint32_t issued = 0;
             bool ok = true;
+            for (int item = blockIdx.x; ok && item < a.items; item += gridDim.x) {
+            int64_t u0, u1;
+            item_range(item, a.splits, a.chunk, a.B, u0, u1);
             for (int64_t u = u0; ok && u < u1; ++u) {
                 const int tile = (int)(u / a.B), i = (int)(u % a.B);
                 const int tm = tile / a.ntn, tn = tile % a.ntn;
@@ -333,6 +359,7 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                     ps.advance(MG_STAGES);
                 }
             }
+            }
             if (!ok) {
                 PipeState q = ps;
                 const uint32_t back = issued < MG_STAGES ? issued : MG_STAGES;
@@ -350,11 +377,12 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             PipeState ps;
             bool ok = true;
             int seg = 0;
+            for (int item = blockIdx.x; ok && item < a.items; item += gridDim.x) {
+            int64_t u0, u1;
+            item_range(item, a.splits, a.chunk, a.B, u0, u1);
             int64_t u = u0;
             while (ok && u < u1) {
-                const int tile = (int)(u / a.B);
-                int64_t u_end = (int64_t)(tile + 1) * a.B;     // end of this tile's samples
-                if (u_end > u1) u_end = u1;
+                const int64_t u_end = u1;                      // an item never crosses a tile
                 if (!mbar_wait(tempty_bar, (seg & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
                 tc_fence_after();
                 bool first = true;
@@ -384,6 +412,7 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                 if (ok) mma_commit(tfull_bar);
                 ++seg;
             }
+            }
             if (!ok) {
                 mma_commit(drain_bar);
                 int never = 0;
@@ -394,13 +423,16 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         const uint32_t q = warp & 3;            // TMEM lane quarter
         const uint32_t half = (warp - 2) >> 2;  // rows 0-127 or 128-255 of the tile
         int seg = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; ok && item < a.items; item += gridDim.x) {
+        int64_t u0, u1;
+        item_range(item, a.splits, a.chunk, a.B, u0, u1);
         int64_t u = u0;
         while (u < u1) {
             const int tile = (int)(u / a.B);
-            int64_t u_end = (int64_t)(tile + 1) * a.B;
-            if (u_end > u1) u_end = u1;
+            const int64_t u_end = u1;
             const int tm = tile / a.ntn, tn = tile % a.ntn;
-            if (!mbar_wait(tfull_bar, seg & 1u, abortp, kWaitLimitNs)) break;
+            if (!mbar_wait(tfull_bar, seg & 1u, abortp, kWaitLimitNs)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((q * 32u) << 16) + half * 256u;
             const int m = tm * MG_BM + (int)half * 128 + (int)q * 32 + lane;
@@ -432,6 +464,231 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             if (lane == 0) mbar_arrive(tempty_bar);
             u = u_end;
             ++seg;
+        }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
+}
+
+// =====================================================================================
+// direct kernel: per-sample weight-gradient tiles formed in TMEM, never written out
+// =====================================================================================
+// For one (128 x 256 output tile, sample i) unit the contraction over the sample's
+// T tokens leaves the tile of G_i = D_i^T X_i in TMEM.  The epilogue squares and
+// sums it into n_i and adds it to a register copy of the tile of S = sum_i G_i,
+// which is flushed to global memory when the CTA moves to another tile.  One GEMM
+// (2 B T d_in d_out flops) thus yields both the per-sample norms and the gradient
+// sum; it beats the Gram route whenever T exceeds d_in d_out / (d_in + d_out).
+constexpr int DR_BM = 128;                          // d_out rows per tile
+constexpr int DR_BN = 256;                          // d_in columns per tile
+constexpr int DR_BK = 64;                           // tokens per stage
+constexpr int DR_STAGES = 4;
+constexpr int DR_BOX_BYTES = 64 * DR_BK * 2;        // 8 KB
+constexpr int DR_A_BYTES = (DR_BM / 64) * DR_BOX_BYTES;
+constexpr int DR_B_BYTES = (DR_BN / 64) * DR_BOX_BYTES;
+constexpr int DR_STAGE_BYTES = DR_A_BYTES + DR_B_BYTES;   // 48 KB
+constexpr int DR_SMEM = DR_STAGES * DR_STAGE_BYTES + 1024 + 256;
+// Epilogue: three warps per TMEM lane quarter; the 16 column chunks (of 16) of a tile
+// row are split 6 / 5 / 5 among them, so a thread keeps at most 96 columns of the S
+// tile in registers (16 warps' worth of register file at 128 registers per thread).
+constexpr int DR_EPI_WARPS = 12;
+constexpr int DR_CHUNKS_MAX = 6;
+constexpr int DR_COLS = DR_CHUNKS_MAX * 16;
+constexpr int DR_THREADS = 64 + 32 * DR_EPI_WARPS;  // warp 0 TMA, warp 1 MMA, the rest epilogue
+
+struct DirectArgs {
+    int B, T, d_in, d_out;
+    int ntm, ntn;
+    int splits, chunk, items;   // see SplitPlan
+    float* n;           // [B], +=
+    float* S;           // [d_out, d_in], += ; may be null
+    int* status;
+};
+
+__global__ void __launch_bounds__(DR_THREADS, 1)
+direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
+                     const DirectArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_base = smem_base + DR_STAGES * DR_STAGE_BYTES;
+    auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (DR_STAGES + s); };
+    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * DR_STAGES + b); };
+    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * DR_STAGES + 2 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * DR_STAGES + 4);
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (uint32_t s = 0; s < DR_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), DR_EPI_WARPS); }
+        mbar_init(drain_bar, 1);
+        fence_barrier_init();
+        prefetch_tmap(&tmX);
+        prefetch_tmap(&tmD);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);   // two 128x256 fp32 accumulators
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    const int kt = (a.T + DR_BK - 1) / DR_BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            PipeState ps;
+            uint32_t issued = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < a.items; item += gridDim.x) {
+            int64_t u0, u1;
+            item_range(item, a.splits, a.chunk, a.B, u0, u1);
+            for (int64_t u = u0; ok && u < u1; ++u) {
+                const int tile = (int)(u / a.B), i = (int)(u % a.B);
+                const int tm = tile / a.ntn, tn = tile % a.ntn;
+                for (int c = 0; c < kt; ++c) {
+                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                    const uint32_t sA = smem_base + ps.stage * DR_STAGE_BYTES;
+                    const uint32_t sB = sA + DR_A_BYTES;
+                    mbar_arrive_expect_tx(full_bar(ps.stage), DR_STAGE_BYTES);
+#pragma unroll
+                    for (int mb = 0; mb < DR_BM / 64; ++mb)
+                        tma_load_3d(sA + mb * DR_BOX_BYTES, &tmD, full_bar(ps.stage), tm * DR_BM + mb * 64, c * DR_BK, i);
+#pragma unroll
+                    for (int nb = 0; nb < DR_BN / 64; ++nb)
+                        tma_load_3d(sB + nb * DR_BOX_BYTES, &tmX, full_bar(ps.stage), tn * DR_BN + nb * 64, c * DR_BK, i);
+                    ++issued;
+                    ps.advance(DR_STAGES);
+                }
+            }
+            }
+            if (!ok) {
+                PipeState q = ps;
+                const uint32_t back = issued < DR_STAGES ? issued : DR_STAGES;
+                for (uint32_t r = 0; r < back; ++r) {
+                    if (q.stage == 0) { q.stage = DR_STAGES - 1; q.phase ^= 1u; } else { --q.stage; }
+                    int never = 0;
+                    mbar_wait(full_bar(q.stage), q.phase, &never, kDrainLimitNs);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(DR_BM, DR_BN, 1, 1);   // both operands MN-major
+            PipeState ps;
+            bool ok = true;
+            int n_unit = 0;
+            for (int item = blockIdx.x; ok && item < a.items; item += gridDim.x) {
+            int64_t u0, u1;
+            item_range(item, a.splits, a.chunk, a.B, u0, u1);
+            for (int64_t u = u0; ok && u < u1; ++u, ++n_unit) {
+                const uint32_t buf = n_unit & 1, use = n_unit >> 1;
+                if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t acc = tmem_base + buf * 256u;
+                for (int c = 0; c < kt; ++c) {
+                    if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, kWaitLimitNs)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sA = smem_base + ps.stage * DR_STAGE_BYTES;
+                    const uint32_t sB = sA + DR_A_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < DR_BK / 16; ++kk) {
+                        const uint64_t da = smem_desc_sw128(sA + kk * 2048, DR_BOX_BYTES, 1024);
+                        const uint64_t db = smem_desc_sw128(sB + kk * 2048, DR_BOX_BYTES, 1024);
+                        mma_bf16(acc, da, db, idesc, (c == 0 && kk == 0) ? 0u : 1u);
+                    }
+                    mma_commit(empty_bar(ps.stage));
+                    ps.advance(DR_STAGES);
+                }
+                if (ok) mma_commit(tfull_bar(buf));
+            }
+            }
+            if (!ok) {
+                mma_commit(drain_bar);
+                int never = 0;
+                mbar_wait(drain_bar, 0, &never, kDrainLimitNs);
+            }
+        }
+    } else {
+        const uint32_t q = warp & 3;            // TMEM lane quarter: rows 32q .. 32q+31 of the tile
+        const uint32_t part = (warp - 2) >> 2;  // which column slice of the tile: chunks [c_begin, c_begin + n_chunks)
+        const int c_begin = part == 0 ? 0 : (part == 1 ? 6 : 11);
+        const int n_chunks = part == 0 ? 6 : 5;
+        float sacc[DR_COLS];                    // this thread's row of the S tile (its column slice)
+#pragma unroll
+        for (int e = 0; e < DR_COLS; ++e) sacc[e] = 0.f;
+        int n_unit = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; ok && item < a.items; item += gridDim.x) {
+        int64_t u0, u1;
+        item_range(item, a.splits, a.chunk, a.B, u0, u1);
+        int64_t u = u0;
+        while (ok && u < u1) {
+            // one segment: this work item's samples of its output tile
+            const int tile = (int)(u / a.B);
+            const int64_t u_end = u1;
+            for (; u < u_end; ++u, ++n_unit) {
+                const int i = (int)(u - (int64_t)tile * a.B);
+                const uint32_t buf = n_unit & 1, use = n_unit >> 1;
+                if (!mbar_wait(tfull_bar(buf), use & 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((q * 32u) << 16) + buf * 256u + (uint32_t)c_begin * 16u;
+                float sq = 0.f;
+#pragma unroll
+                for (int cc = 0; cc < DR_CHUNKS_MAX; ++cc) {
+                    if (cc < n_chunks) {             // uniform across the warp
+                        uint32_t r[16];
+                        tmem_ld16(taddr + cc * 16, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const float v = __uint_as_float(r[e]);
+                            sq = fmaf(v, v, sq);
+                            sacc[cc * 16 + e] += v;
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(buf));
+                const float w = warp_sum_f(sq);
+                if (lane == 0) atomicAdd(a.n + i, w);
+            }
+            // end of the segment: add this thread's part of the tile's row into S
+            const int tm = tile / a.ntn, tn = tile % a.ntn;
+            const int m = tm * DR_BM + (int)q * 32 + lane;
+            const int n0 = tn * DR_BN + c_begin * 16;
+            float* srow = a.S + (int64_t)m * a.d_in;
+            const bool row_ok = ok && a.S != nullptr && m < a.d_out;
+#pragma unroll
+            for (int e = 0; e < DR_COLS; e += 4) {
+                const int n = n0 + e;
+                if (row_ok && e < n_chunks * 16) {
+                    if (n + 3 < a.d_in) {
+                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(srow + n),
+                                     "f"(sacc[e]), "f"(sacc[e + 1]), "f"(sacc[e + 2]), "f"(sacc[e + 3]) : "memory");
+                    } else {
+#pragma unroll
+                        for (int z = 0; z < 4; ++z)
+                            if (n + z < a.d_in) atomicAdd(srow + n + z, sacc[e + z]);
+                    }
+                }
+                sacc[e] = 0.f; sacc[e + 1] = 0.f; sacc[e + 2] = 0.f; sacc[e + 3] = 0.f;
+            }
+        }
         }
     }
 
@@ -528,8 +785,9 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
     a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
     a.ntm = (int)((d_out + MG_BM - 1) / MG_BM);
     a.ntn = (int)((d_in + MG_BN - 1) / MG_BN);
-    a.units = (int64_t)a.ntm * a.ntn * B;
-    if (a.units / B > 0x7fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    if ((int64_t)a.ntm * a.ntn * B > 0x3fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    const SplitPlan sp = make_split((int64_t)a.ntm * a.ntn, B, ctx->sm_count);
+    a.splits = sp.splits; a.chunk = sp.chunk; a.items = sp.items;
     a.S = S; a.status = ctx->gemm_status;
     if (!accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
     static bool attr_set = false;
@@ -537,8 +795,38 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
         ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(mean_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM));
         attr_set = true;
     }
-    const int grid = a.units < ctx->sm_count ? (int)a.units : ctx->sm_count;
+    const int grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
     mean_grad_kernel<<<grid, MG_THREADS, MG_SMEM, st>>>(tmX, tmD, a);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                         int64_t d_out, float* n, int accumulate_norms, float* S, int accumulate_sum,
+                         cudaStream_t st) {
+    CUtensorMap tmX, tmD;
+    int rc = make_map(ctx, &tmX, X, B, T, d_in, DR_BK);
+    if (rc != ADLOCO_OK) return rc;
+    rc = make_map(ctx, &tmD, D, B, T, d_out, DR_BK);
+    if (rc != ADLOCO_OK) return rc;
+    DirectArgs a;
+    a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
+    a.ntm = (int)((d_out + DR_BM - 1) / DR_BM);
+    a.ntn = (int)((d_in + DR_BN - 1) / DR_BN);
+    if ((int64_t)a.ntm * a.ntn * B > 0x3fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    const SplitPlan sp = make_split((int64_t)a.ntm * a.ntn, B, ctx->sm_count);
+    a.splits = sp.splits; a.chunk = sp.chunk; a.items = sp.items;
+    a.n = n; a.S = S; a.status = ctx->gemm_status;
+    if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
+    if (S && !accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
+    static bool attr_set = false;
+    if (!attr_set) {
+        ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(direct_sqnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_SMEM));
+        attr_set = true;
+    }
+    const int grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
+    direct_sqnorm_kernel<<<grid, DR_THREADS, DR_SMEM, st>>>(tmX, tmD, a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;

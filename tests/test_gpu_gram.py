@@ -23,19 +23,26 @@ def ctx():
     c.close()
 
 
-def _gpu_layer(ctx, X, D, want_S=True):
+def _gpu_layer(ctx, X, D, want_S=True, method="gram"):
     B = X.shape[0]
     n = torch.full((B,), -5.0, device=DEV)
     S = torch.full((D.shape[2], X.shape[2]), -5.0, device=DEV) if want_S else None
-    ctx.gram_sqnorm(X, D, n, grad_sum=S)
+    if method == "gram":
+        ctx.gram_sqnorm(X, D, n, grad_sum=S)
+    else:
+        ctx.linear_sqnorm(X, D, n, grad_sum=S, method=method)
     torch.cuda.synchronize()
     return n, S
 
 
-def test_small_integer_layer_is_exact(ctx):
+METHODS = ["gram", "direct", "auto"]
+
+
+@pytest.mark.parametrize("method", METHODS)
+def test_small_integer_layer_is_exact(ctx, method):
     # every product and partial sum is an integer below 2^24: the result must be exact
     X, D = W.small_integer_layer(3, 5, 8, 16, seed=9, device=DEV)
-    n, S = _gpu_layer(ctx, X, D)
+    n, S = _gpu_layer(ctx, X, D, method=method)
     n_ref, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
     assert np.array_equal(n.cpu().numpy().astype(np.float64), n_ref)
     assert np.array_equal(S.cpu().numpy().astype(np.float64), S_ref)
@@ -50,9 +57,10 @@ def test_small_integer_layer_is_exact(ctx):
     (4, 130, 264, 520),      # d_in > 256 and d_out > 512: several output tiles, ragged
     (33, 64, 32, 48),
 ])
-def test_layer_matches_oracle(ctx, B, T, d_in, d_out):
+@pytest.mark.parametrize("method", METHODS)
+def test_layer_matches_oracle(ctx, B, T, d_in, d_out, method):
     X, D = W.linear_layer(B, T, d_in, d_out, seed=B + T, device=DEV)
-    n, S = _gpu_layer(ctx, X, D)
+    n, S = _gpu_layer(ctx, X, D, method=method)
     n_ref, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
     assert np.allclose(n.cpu().numpy(), n_ref, rtol=TOL_BF16, atol=0), (n.cpu().numpy() / n_ref)
     scale = np.abs(S_ref).max()
@@ -81,6 +89,25 @@ def test_accumulate_flags_and_unsupported_shapes(ctx):
     with pytest.raises(A.AdlocoError) as e:
         ctx.gram_sqnorm(Xb, Db, n3)
     assert e.value.status == A.ERR_UNSUPPORTED and ctx.launch_count == before
+
+
+def test_direct_route_accumulates_and_may_skip_the_sum(ctx):
+    X, D = W.linear_layer(3, 200, 72, 264, seed=4, device=DEV)
+    n, S = _gpu_layer(ctx, X, D, method="direct")
+    n2, S2 = n.clone(), S.clone()
+    ctx.linear_sqnorm(X, D, n2, accumulate_norms=True, grad_sum=S2, accumulate_sum=True, method="direct")
+    n3 = torch.zeros(3, device=DEV)
+    ctx.linear_sqnorm(X, D, n3, method="direct")              # no sum buffer
+    torch.cuda.synchronize()
+    assert torch.allclose(n2, 2 * n, rtol=1e-5) and torch.allclose(S2, 2 * S, rtol=1e-5, atol=1e-5 * float(S.abs().max()))
+    assert torch.allclose(n3, n, rtol=1e-5)
+    ng, Sg = _gpu_layer(ctx, X, D, method="gram")            # the two routes agree with each other as well
+    assert torch.allclose(ng, n, rtol=2e-3) and torch.allclose(Sg, S, rtol=1e-4, atol=1e-4 * float(S.abs().max()))
+    with pytest.raises(A.AdlocoError) as e:
+        ctx.lib.adloco_linear_sqnorm  # noqa: B018  (symbol exists)
+        ctx.check(ctx.lib.adloco_linear_sqnorm(ctx.h, X.data_ptr(), D.data_ptr(), 3, 200, 72, 264, n.data_ptr(), 0,
+                                               None, 0, 7, None), "adloco_linear_sqnorm")
+    assert e.value.status == A.ERR_INVALID_ARG
 
 
 def test_whole_model_switch_mode_small(ctx):
