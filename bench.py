@@ -396,6 +396,172 @@ def run_ours(args, rank, world, local_rank):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------------
+# per-configuration table (python bench.py --table): one JSON line per row
+# ------------------------------------------------------------------------------------
+def run_table(args):
+    """Times every kernel of the five workload configurations on one GPU, with the
+    oracle beside it (whole where it finishes in seconds, else on a stated sample and
+    extrapolated).  Configurations whose inputs fit in L2 are timed with an L2 flush
+    (a 512 MB write) between repetitions."""
+    import numpy as np
+    import oracle.adloco_oracle as O
+    from paper_2508_18182_b200 import binding as A
+    from paper_2508_18182_b200.build import build
+
+    build()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = A.Context(0)
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream()
+    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+
+    def gpu_ms(fn, reps=20, flush=False, warm=3):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            if flush:
+                flush_buf.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        ts.sort()
+        return ts[len(ts) // 2]
+
+    def cpu_s(fn):
+        t0 = time.perf_counter()
+        fn()
+        return time.perf_counter() - t0
+
+    def emit(config, kernel, ms, *, nbytes=None, flops=None, oracle_s=None, oracle_note="", note=""):
+        row = {"config": config, "kernel": kernel, "gpu_ms": round(ms, 4)}
+        if nbytes is not None:
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            row.update({"algorithmic_bytes": nbytes, "GB/s": round(gbs, 1),
+                        "frac_measured_hbm": round(gbs / peaks["hbm_gbs"], 3), "frac_nominal_8TBs": round(gbs / 8000, 3)})
+        if flops is not None:
+            tf = flops / (ms * 1e-3) / 1e12
+            row.update({"algorithmic_flops": flops, "TFLOP/s": round(tf, 1),
+                        "frac_measured_bf16": round(tf / peaks["bf16_tflops"], 3), "frac_nominal_2250": round(tf / 2250, 3)})
+        if oracle_s is not None:
+            row.update({"oracle_s": round(oracle_s, 3), "oracle_note": oracle_note,
+                        "speedup": round(oracle_s / (ms * 1e-3), 1)})
+        if note:
+            row["note"] = note
+        print(json.dumps(row), flush=True)
+
+    def outer_case(config, K, P, dtype):
+        theta, inst, mom = W.outer_state(K, P, inst_dtype=dtype, seed=7, device=dev)
+        es = 2 if dtype == torch.bfloat16 else 4
+        ms = gpu_ms(lambda: ctx.outer_step(inst, theta, mom, lr=LR, momentum=MU), flush=(P * (es * K + 16) < (1 << 29)))
+        sl = min(P, 1 << 24)
+        th, v, ins = W.to_numpy(theta[:sl]), W.to_numpy(mom[:sl]), [W.to_numpy(t[:sl]) for t in inst]
+        o_s = cpu_s(lambda: O.outer_step(th, ins, v, lr=LR, momentum=MU)) * (P / sl)
+        emit(config, f"outer_step (K={K} {'bf16' if es == 2 else 'fp32'}, P={P})", ms, nbytes=(es * K + 16) * P,
+             oracle_s=o_s, oracle_note="whole" if sl == P else f"timed on {sl} elements, extrapolated")
+        del theta, inst, mom
+
+    # config 1
+    G = W.per_sample_grads(16, 1 << 20, seed=1, device=dev)
+    p = A.make_params(0.5, b_cur=16, b_max=32)
+    ms = gpu_ms(lambda: ctx.norm_test(G, p, sync=False), flush=True)
+    Gn = W.to_numpy(G)
+    emit(1, "norm_test (B=16, P=2^20)", ms, nbytes=4 * 16 * (1 << 20), oracle_s=cpu_s(lambda: O.norm_test(Gn, eta=0.5)),
+         oracle_note="whole", note="L2 flushed between repetitions; launch-latency bound")
+    outer_case(1, 4, 1 << 20, torch.float32)
+    del G
+    # config 2
+    G = W.per_sample_grads(NT_B, 1 << 24, seed=2, device=dev)
+    p = A.make_params(0.1, b_cur=64, b_max=32)
+
+    def c2():
+        ctx.norm_test(G, p, sync=False)
+        ctx.test_decide(A.make_params(0.5, b_cur=64, b_max=32), sync=False)
+        ctx.test_decide(A.make_params(1.0, b_cur=64, b_max=32), sync=False)
+    ms = gpu_ms(c2)
+    Gn = W.to_numpy(G)
+    emit(2, "norm_test + eta sweep (B=64, P=2^24)", ms, nbytes=4 * 64 * (1 << 24),
+         oracle_s=cpu_s(lambda: O.norm_test(Gn, eta=0.1)), oracle_note="whole")
+    del G, Gn
+    outer_case(2, 8, W.GPT2_SMALL_P, torch.bfloat16)
+    # config 3
+    X, D = W.linear_layer(GR_B, GR_T, GR_DIN, GR_DOUT, seed=3, device=dev)
+    n = torch.zeros(GR_B, device=dev)
+    S = torch.zeros(GR_DOUT, GR_DIN, device=dev)
+    sym, executed, mg = gram_flops()
+    ms_g = gpu_ms(lambda: ctx.gram_sqnorm(X, D, n))
+    ms_gs = gpu_ms(lambda: ctx.gram_sqnorm(X, D, n, grad_sum=S))
+    ms_d = gpu_ms(lambda: ctx.linear_sqnorm(X, D, n, grad_sum=S, method="direct"))
+    Xn, Dn = W.to_numpy(X), W.to_numpy(D)
+    o_s = cpu_s(lambda: O.linear_layer_terms(Xn, Dn))
+    emit(3, "gram_sqnorm (norms only)", ms_g, flops=sym, note=f"executed {executed / (ms_g * 1e-3) / 1e12:.0f} TFLOP/s")
+    emit(3, "gram_sqnorm + mean-gradient GEMM", ms_gs, flops=sym + mg, oracle_s=o_s, oracle_note="whole (BLAS dgemm per sample)")
+    emit(3, "mean-gradient GEMM (difference)", ms_gs - ms_g, flops=mg)
+    emit(3, "linear_sqnorm direct (norms + gradient sum)", ms_d, flops=mg, oracle_s=o_s, oracle_note="whole",
+         note="same outputs as the row above from one GEMM")
+    # config 4: 12 blocks x 4 layers x 4 micro-batches, all inputs resident (38.7 GB)
+    shapes = list(W.GPT2_SMALL_BLOCK_LINEARS) * 12
+    data = [[W.linear_layer(32, 1024, di, do, seed=1000 * j + l, device=dev) for l, (di, do) in enumerate(shapes)]
+            for j in range(4)]
+    sums = [torch.zeros(do, di, device=dev) for di, do in shapes]
+    acc = A.Accumulator(ctx, sums)
+    n_mb = torch.zeros(32, device=dev)
+    p4 = A.make_params(0.5, b_cur=128, b_max=32)
+
+    def whole_model(method):
+        acc.reset()
+        for j in range(4):
+            for l, (Xl, Dl) in enumerate(data[j]):
+                if method == "gram":
+                    ctx.gram_sqnorm(Xl, Dl, n_mb, accumulate_norms=(l > 0), grad_sum=sums[l], accumulate_sum=True)
+                else:
+                    ctx.linear_sqnorm(Xl, Dl, n_mb, accumulate_norms=(l > 0), grad_sum=sums[l], accumulate_sum=True,
+                                      method=method)
+            acc.accumulate(per_sample_sqnorm=n_mb)
+        acc.finalize(p4, sync=False)
+    f_sym = sum(32 * 1024 * 1025 * (di + do) for di, do in shapes) * 4
+    f_mg = sum(2 * 32 * 1024 * di * do for di, do in shapes) * 4
+    ms4 = gpu_ms(lambda: whole_model("gram"), reps=5, warm=1)
+    Xb = [(W.to_numpy(data[0][l][0]), W.to_numpy(data[0][l][1])) for l in range(4)]
+    o4 = cpu_s(lambda: [O.linear_layer_terms(x, d) for x, d in Xb]) * 48
+    emit(4, "whole model, Gram route (48 layers x 4 micro-batches + finalize)", ms4, flops=f_sym + f_mg, oracle_s=o4,
+         oracle_note="one block x one micro-batch timed, x48 extrapolated")
+    ms4d = gpu_ms(lambda: whole_model("auto"), reps=5, warm=1)
+    emit(4, "whole model, linear_sqnorm auto (direct route)", ms4d, flops=f_mg, oracle_s=o4, oracle_note="as above")
+    acc.close()
+    del data, sums
+    torch.cuda.empty_cache()
+    # config 5
+    outer_case(5, 4, W.LARGE_P, torch.bfloat16)
+    mbs = W.micro_batches(8, 32, 1 << 22, sigma=1.0, mean_scale="raw", seed=5, device=dev)
+    Sacc = torch.zeros(1 << 22, device=dev)
+    acc = A.Accumulator(ctx, [Sacc])
+    p5 = A.make_params(0.5, b_cur=256, b_max=32)
+
+    def c5():
+        acc.reset()
+        for m in mbs:
+            acc.accumulate(m)
+        acc.finalize(p5, sync=False)
+    ms = gpu_ms(c5, reps=10)
+    mbn = [W.to_numpy(m) for m in mbs]
+    emit(5, "accumulate x8 + finalize (B=256, P=2^22)", ms, nbytes=8 * (4 * 32 + 8) * (1 << 22),
+         oracle_s=cpu_s(lambda: O.accumulated_norm_test(mbn, eta=0.5)), oracle_note="whole")
+    acc.close()
+    # trainer merge
+    _, inst, _ = W.outer_state(4, W.GPT2_SMALL_P, inst_dtype=torch.bfloat16, seed=9, device=dev)
+    out = torch.empty_like(inst[0])
+    ms = gpu_ms(lambda: ctx.merge(inst, [3, 17, 5, 8], out))
+    emit("merge", "adloco_merge (K=4 bf16, P=124,439,808)", ms, nbytes=(2 * 4 + 2) * W.GPT2_SMALL_P)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -404,6 +570,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--table", action="store_true", help="per-configuration table, one JSON line per row")
     ap.add_argument("--small", action="store_true",
                     help="profiling case: same kernels on inputs of a few hundred MB (not a bench value)")
     args = ap.parse_args()
@@ -415,6 +582,10 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.table:
+        if rank == 0:
+            run_table(args)
         return
     if world > 1:
         import torch.distributed as dist
