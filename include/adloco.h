@@ -114,6 +114,16 @@ const char* adloco_last_cuda_error(const adloco_ctx* ctx);
 /* Number of kernel launches this ctx has enqueued so far. */
 int64_t adloco_launch_count(const adloco_ctx* ctx);
 
+/* The tensor-core kernels wait on hardware barriers (tile arrived, accumulator
+ * drained).  Every such wait is bounded: when `limit_ns` of wall time pass the
+ * kernel stops waiting, lets its copies in flight land, frees its tensor memory,
+ * returns, and raises the context's device status word to ADLOCO_ERR_TIMEOUT; the
+ * outputs of that call are then undefined but the context stays usable.  Default
+ * 2 s.  adloco_device_status reads the word (synchronises `stream`) and
+ * optionally clears it. */
+int adloco_set_wait_limit(adloco_ctx* ctx, uint64_t limit_ns);
+int adloco_device_status(adloco_ctx* ctx, int32_t* status_host, int clear, void* stream);
+
 /* ---- norm test on materialised per-sample gradients ---------------------- */
 
 /* Section "Norm test" (Eq. 1, sigma^2_B, b_{k+1}) followed by the switch-mode
@@ -231,7 +241,9 @@ int adloco_accumulate(adloco_ctx* ctx, adloco_accum* acc, const void* grads, adl
 
 /* One test on everything accumulated: N = sum_bufs ||S/b||^2,
  * V = centred_ss/(b-ddof) when every micro-batch was materialised, otherwise
- * V = (Q - b N)/(b - ddof); then the batch rule and switch plan. */
+ * V = (Q - b N)/(b - ddof); then the batch rule and switch plan.  ||S||^2 is taken
+ * from the last form-(a) call when that was the last change to S (the caller must
+ * not modify S behind a form-(a) accumulation), else reduced here. */
 int adloco_accum_finalize(adloco_ctx* ctx, adloco_accum* acc, const adloco_test_params* params,
                           adloco_test_sums* sums_dev, adloco_test_result* result_dev,
                           adloco_test_result* result_host, void* stream);

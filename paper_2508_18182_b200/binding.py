@@ -22,6 +22,7 @@ FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN = 1, 2, 4, 8
 # every symbol that include/adloco.h declares
 EXPORTS = (
     "adloco_create", "adloco_destroy", "adloco_status_string", "adloco_last_cuda_error", "adloco_launch_count",
+    "adloco_set_wait_limit", "adloco_device_status",
     "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_gram_sqnorm", "adloco_linear_sqnorm",
     "adloco_accum_create", "adloco_accum_reset", "adloco_accum_destroy", "adloco_accumulate",
     "adloco_accum_finalize", "adloco_outer_step", "adloco_outer_step_host", "adloco_check_merge", "adloco_merge",
@@ -75,6 +76,8 @@ def load_library() -> C.CDLL:
         "adloco_status_string": (C.c_char_p, [C.c_int]),
         "adloco_last_cuda_error": (C.c_char_p, [vp]),
         "adloco_launch_count": (i64, [vp]),
+        "adloco_set_wait_limit": (C.c_int, [vp, C.c_uint64]),
+        "adloco_device_status": (C.c_int, [vp, C.POINTER(C.c_int32), C.c_int, vp]),
         "adloco_norm_test": (C.c_int, [vp, vp, C.c_int, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp, vp, vp, vp]),
         "adloco_test_decide": (C.c_int, [vp, vp, C.POINTER(TestParams), vp, vp, vp]),
         "adloco_norm_test_host": (C.c_int, [vp, vp, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp]),
@@ -155,6 +158,14 @@ class Context:
             if rc == ERR_CUDA:
                 msg += ": " + self.lib.adloco_last_cuda_error(self.h).decode()
             raise AdlocoError(rc, f"{what}: {msg}")
+
+    def set_wait_limit(self, limit_ns: int):
+        self.check(self.lib.adloco_set_wait_limit(self.h, int(limit_ns)), "adloco_set_wait_limit")
+
+    def device_status(self, clear: bool = True, stream=None) -> int:
+        v = C.c_int32(0)
+        self.check(self.lib.adloco_device_status(self.h, C.byref(v), int(clear), _stream(stream)), "adloco_device_status")
+        return v.value
 
     @property
     def launch_count(self) -> int:

@@ -115,6 +115,24 @@ int adloco_destroy(adloco_ctx* ctx) {
     return ADLOCO_OK;
 }
 
+int adloco_set_wait_limit(adloco_ctx* ctx, uint64_t limit_ns) {
+    if (!ctx) return ADLOCO_ERR_INVALID_ARG;
+    ctx->wait_limit_ns = limit_ns;
+    return ADLOCO_OK;
+}
+
+int adloco_device_status(adloco_ctx* ctx, int32_t* status_host, int clear, void* stream) {
+    if (!ctx || !status_host) return ADLOCO_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int v = 0;
+    ADLOCO_CUDA_TRY(ctx, cudaMemcpyAsync(&v, ctx->gemm_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    if (clear) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(ctx->gemm_status, 0, sizeof(int), st));
+    ADLOCO_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+    *status_host = v;
+    return ADLOCO_OK;
+}
+
 // ---------------------------------------------------------------------------------
 // norm test
 // ---------------------------------------------------------------------------------
@@ -328,6 +346,7 @@ int adloco_accum_reset(adloco_ctx* ctx, adloco_accum* a, void* stream) {
     for (int i = 0; i < a->n_bufs; ++i)
         ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(a->bufs_host[i], 0, (size_t)a->sizes_host[i] * sizeof(float), st));
     ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(a->state, 0, sizeof(adloco_test_sums), st));
+    a->sqnorm_current = true;
     return ADLOCO_OK;
 }
 
@@ -338,6 +357,7 @@ int adloco_accumulate(adloco_ctx* ctx, adloco_accum* a, const void* grads, adloc
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (grads == nullptr) {
         if (!per_sample_sqnorm) return ADLOCO_ERR_INVALID_ARG;
+        a->sqnorm_current = false;   // the caller has changed the S buffers itself
         return launch_accum_add_norms(ctx, a, per_sample_sqnorm, b_micro, st);
     }
     int rc = check_grads(grads, dtype, b_micro, P, row_stride);
@@ -348,6 +368,8 @@ int adloco_accumulate(adloco_ctx* ctx, adloco_accum* a, const void* grads, adloc
     l.B = b_micro; l.P = P; l.stride = row_stride;
     l.n_out = per_sample_sqnorm; l.S = a->bufs_host[0];
     l.sums = a->state; l.result = nullptr; l.mode = NT_MICRO;
+    // this pass rewrites all of S and leaves ||S||^2 in the state
+    a->sqnorm_current = true;
     return launch_norm_test(ctx, l, st);
 }
 
@@ -359,10 +381,12 @@ int adloco_accum_finalize(adloco_ctx* ctx, adloco_accum* a, const adloco_test_pa
     if (rc != ADLOCO_OK) return rc;
     DeviceGuard g(ctx->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // ||S||^2 over every buffer (the materialised form keeps it current, but the
-    // buffers may also have been filled by the tensor-core path)
-    rc = launch_accum_sqnorm(ctx, a, st);
-    if (rc != ADLOCO_OK) return rc;
+    // ||S||^2 over every buffer, unless the last materialised micro-batch left it current
+    if (!a->sqnorm_current) {
+        rc = launch_accum_sqnorm(ctx, a, st);
+        if (rc != ADLOCO_OK) return rc;
+        a->sqnorm_current = true;
+    }
     rc = launch_decide(ctx, a->state, *params, result_dev, st);
     if (rc != ADLOCO_OK) return rc;
     if (sums_dev)

@@ -44,6 +44,7 @@ struct adloco_ctx {
     int max_grid = 0;
     adloco_test_sums* scratch_sums = nullptr;  // used when the caller passes no sums_dev
     int* gemm_status = nullptr;                // device status word of the tensor-core kernels
+    uint64_t wait_limit_ns = 2000000000ull;    // bound of every in-kernel wait: 2 s, far beyond any legitimate wait
     float* n_scratch = nullptr;                // [kMaxBatchRows] per-sample norms when the caller wants none
 
     adloco::HostStaging staging;
@@ -62,6 +63,7 @@ struct adloco_accum {
     int64_t* sizes_dev = nullptr;
     int64_t total_chunks = 0;
     adloco_test_sums* state = nullptr; // device: Q, ||S||^2, centred ss, count
+    bool sqnorm_current = true;        // state->sum_sq_gsum already equals ||S||^2 (kept by the materialised form)
 };
 
 namespace adloco {

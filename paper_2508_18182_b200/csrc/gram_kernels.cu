@@ -20,7 +20,6 @@ namespace adloco {
 
 using namespace ptx;
 
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
 constexpr uint64_t kDrainLimitNs = 50000000ull;    // 50 ms per barrier while leaving after a time-out
 
 struct PipeState {
@@ -62,6 +61,7 @@ struct GramArgs {
     int total_items;
     float* n;             // [B], += (zeroed by the launcher unless accumulating)
     int* status;
+    uint64_t wait_ns;   // bound of every in-kernel wait
 };
 
 __device__ __forceinline__ void gram_decode(int item, const GramArgs& a, int& i, int& ti, int& c0, int& ncb) {
@@ -136,7 +136,7 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 // on the diagonal the row tile is the first column block: fetch it once
                 const bool diag = (c0 == ti);
                 for (int c = 0; c < chunks; ++c) {
-                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
                     const bool is_x = c < kx;
                     const CUtensorMap* map = is_x ? &tmX : &tmD;
                     const int k0 = (is_x ? c : c - kx) * GR_BK;
@@ -172,10 +172,10 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 gram_decode(item, a, i, ti, c0, ncb);
                 const uint32_t idesc = idesc_bf16_f32(GR_TILE, GR_TILE * ncb, 0, 0);
                 // the single accumulator pair must have been drained by the epilogue
-                if (!mbar_wait(tempty_bar, (n_item & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                if (!mbar_wait(tempty_bar, (n_item & 1u) ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 for (int c = 0; c < chunks; ++c) {
-                    if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, kWaitLimitNs)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, a.wait_ns)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t acc = tmem_base + (c < kx ? 0u : 256u);
                     const bool first = (c == 0 || c == kx);
@@ -208,7 +208,8 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         for (int item = blockIdx.x; item < a.total_items; item += gridDim.x, ++n_item) {
             int i, ti, c0, ncb;
             gram_decode(item, a, i, ti, c0, ncb);
-            if (!mbar_wait(tfull_bar, n_item & 1u, abortp, kWaitLimitNs)) break;
+            // the whole warp takes the same decision: the TMEM loads below are warp-collective
+            if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar, n_item & 1u, abortp, a.wait_ns))) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((q * 32u) << 16);
             const int cols_per_half = 64 * ncb;
@@ -294,6 +295,7 @@ struct MeanGradArgs {
     int splits, chunk, items;   // see SplitPlan
     float* S;           // [d_out, d_in], += (zeroed by the launcher unless accumulating)
     int* status;
+    uint64_t wait_ns;   // bound of every in-kernel wait
 };
 
 __global__ void __launch_bounds__(MG_THREADS, 1)
@@ -345,7 +347,7 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                 const int tile = (int)(u / a.B), i = (int)(u % a.B);
                 const int tm = tile / a.ntn, tn = tile % a.ntn;
                 for (int c = 0; c < kt; ++c) {
-                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
                     const uint32_t sA = smem_base + ps.stage * MG_STAGE_BYTES;
                     const uint32_t sB = sA + MG_A_BYTES;
                     mbar_arrive_expect_tx(full_bar(ps.stage), MG_STAGE_BYTES);
@@ -383,12 +385,12 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             int64_t u = u0;
             while (ok && u < u1) {
                 const int64_t u_end = u1;                      // an item never crosses a tile
-                if (!mbar_wait(tempty_bar, (seg & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                if (!mbar_wait(tempty_bar, (seg & 1u) ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 bool first = true;
                 for (; ok && u < u_end; ++u) {
                     for (int c = 0; c < kt; ++c) {
-                        if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, kWaitLimitNs)) { ok = false; break; }
+                        if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, a.wait_ns)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t sA = smem_base + ps.stage * MG_STAGE_BYTES;
                         const uint32_t sB = sA + MG_A_BYTES;
@@ -432,7 +434,7 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             const int tile = (int)(u / a.B);
             const int64_t u_end = u1;
             const int tm = tile / a.ntn, tn = tile % a.ntn;
-            if (!mbar_wait(tfull_bar, seg & 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar, seg & 1u, abortp, a.wait_ns))) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((q * 32u) << 16) + half * 256u;
             const int m = tm * MG_BM + (int)half * 128 + (int)q * 32 + lane;
@@ -510,6 +512,7 @@ struct DirectArgs {
     float* n;           // [B], +=
     float* S;           // [d_out, d_in], += ; may be null
     int* status;
+    uint64_t wait_ns;   // bound of every in-kernel wait
 };
 
 __global__ void __launch_bounds__(DR_THREADS, 1)
@@ -560,7 +563,7 @@ direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const int tile = (int)(u / a.B), i = (int)(u % a.B);
                 const int tm = tile / a.ntn, tn = tile % a.ntn;
                 for (int c = 0; c < kt; ++c) {
-                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
                     const uint32_t sA = smem_base + ps.stage * DR_STAGE_BYTES;
                     const uint32_t sB = sA + DR_A_BYTES;
                     mbar_arrive_expect_tx(full_bar(ps.stage), DR_STAGE_BYTES);
@@ -596,11 +599,11 @@ direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             item_range(item, a.splits, a.chunk, a.B, u0, u1);
             for (int64_t u = u0; ok && u < u1; ++u, ++n_unit) {
                 const uint32_t buf = n_unit & 1, use = n_unit >> 1;
-                if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t acc = tmem_base + buf * 256u;
                 for (int c = 0; c < kt; ++c) {
-                    if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, kWaitLimitNs)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, a.wait_ns)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sA = smem_base + ps.stage * DR_STAGE_BYTES;
                     const uint32_t sB = sA + DR_A_BYTES;
@@ -643,7 +646,7 @@ direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             for (; u < u_end; ++u, ++n_unit) {
                 const int i = (int)(u - (int64_t)tile * a.B);
                 const uint32_t buf = n_unit & 1, use = n_unit >> 1;
-                if (!mbar_wait(tfull_bar(buf), use & 1u, abortp, kWaitLimitNs)) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abortp, a.wait_ns))) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((q * 32u) << 16) + buf * 256u + (uint32_t)c_begin * 16u;
                 float sq = 0.f;
@@ -760,7 +763,7 @@ int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     a.half_per_sample = (int)halves;
     a.n_full = (int)(fulls * B);
     a.total_items = (int)((fulls + halves) * B);
-    a.n = n; a.status = ctx->gemm_status;
+    a.n = n; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
     static bool attr_set = false;
     if (!attr_set) {
@@ -788,7 +791,7 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
     if ((int64_t)a.ntm * a.ntn * B > 0x3fffffff) return ADLOCO_ERR_UNSUPPORTED;
     const SplitPlan sp = make_split((int64_t)a.ntm * a.ntn, B, ctx->sm_count);
     a.splits = sp.splits; a.chunk = sp.chunk; a.items = sp.items;
-    a.S = S; a.status = ctx->gemm_status;
+    a.S = S; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
     static bool attr_set = false;
     if (!attr_set) {
@@ -817,7 +820,7 @@ int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
     if ((int64_t)a.ntm * a.ntn * B > 0x3fffffff) return ADLOCO_ERR_UNSUPPORTED;
     const SplitPlan sp = make_split((int64_t)a.ntm * a.ntn, B, ctx->sm_count);
     a.splits = sp.splits; a.chunk = sp.chunk; a.items = sp.items;
-    a.n = n; a.S = S; a.status = ctx->gemm_status;
+    a.n = n; a.S = S; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
     if (S && !accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
     static bool attr_set = false;

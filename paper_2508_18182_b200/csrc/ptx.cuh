@@ -56,9 +56,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                                           uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;
+    const uint32_t check_mask = limit_ns < 1000 ? 0u : 0xffu;   // look at the clock every 256 polls (every poll for sub-us limits)
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 0xffu) == 0) {
+        if ((it & check_mask) == 0) {
             if (*abort_flag) return false;
             const uint64_t now = globaltimer_ns();
             if (t0 == 0) t0 = now;

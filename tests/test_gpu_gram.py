@@ -136,3 +136,27 @@ def test_whole_model_switch_mode_small(ctx):
     assert_test_result(r, ora, p, TOL_BF16, stat_tol=TOL_BF16 * max(1.0, kappa), what="whole model")
     assert r.flags & A.FLAG_ACCUMULATE
     acc.close()
+
+
+@pytest.mark.parametrize("method", METHODS[:2])
+def test_a_wait_that_runs_out_raises_the_status_and_the_context_stays_usable(method):
+    """Every in-kernel wait is bounded.  With the bound set to one nanosecond the
+    first wait that is not satisfied at once gives up: the kernel must leave through
+    its teardown (copies landed, tensor memory freed), raise ADLOCO_ERR_TIMEOUT in the
+    status word, and the next call with the normal bound must be correct again."""
+    c = A.Context(0)
+    X, D = W.linear_layer(8, 512, 256, 512, seed=77, device=DEV)
+    n = torch.zeros(8, device=DEV)
+    S = torch.zeros(512, 256, device=DEV)
+    assert c.device_status() == 0
+    c.set_wait_limit(1)
+    c.linear_sqnorm(X, D, n, grad_sum=S, method=method)
+    assert c.device_status(clear=True) == A.ERR_TIMEOUT
+    assert c.device_status() == 0
+    c.set_wait_limit(2_000_000_000)
+    c.linear_sqnorm(X, D, n, grad_sum=S, method=method)
+    assert c.device_status() == 0
+    n_ref, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
+    assert np.allclose(n.cpu().numpy(), n_ref, rtol=TOL_BF16)
+    assert np.allclose(S.cpu().numpy(), S_ref, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(S_ref).max() * 0.05)
+    c.close()
