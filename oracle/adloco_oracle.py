@@ -163,6 +163,79 @@ def norm_test(G, *, eta: float, ddof: int = 1, b_cur: int = 1, b_max: int = 1,
 
 
 # --------------------------------------------------------------------------
+# inner-product test and augmented inner-product test
+# --------------------------------------------------------------------------
+@dataclass
+class InnerProductResult:
+    var_ip: float = 0.0        # Var_i <g_i, gbar>
+    stat_ip: float = 0.0       # var_ip / (theta^2 ||gbar||^4)
+    var_orth: float = 0.0      # Var_i of the component of g_i orthogonal to gbar
+    stat_orth: float = 0.0     # var_orth / (nu^2 ||gbar||^2)
+    mean_sqnorm: float = 0.0
+    batch_count: int = 0
+    b_ip: int = 1
+    b_aug: int = 1
+    flags: int = 0
+    inner_products: np.ndarray = field(default_factory=lambda: np.zeros(0))
+
+
+def inner_product_tests(G, *, theta: float, nu: float, ddof: int = 1, b_cur: int = 1,
+                        b_cap: int = 0) -> InnerProductResult:
+    """Inner-product test and its augmented form (Section "Inner product test").
+
+    p_i      = <g_i, gbar>
+    b_ip     = ceil( Var_i(p_i) / (theta^2 ||gbar||^4) )
+    o_i      = g_i - (p_i / ||gbar||^2) gbar            (component orthogonal to gbar)
+    b_aug    = ceil( max{ b_ip, Var_i(o_i) / (nu^2 ||gbar||^2) } )
+    Variances use the (b - ddof) normaliser; the variance of the vectors o_i is
+    the trace of their sample covariance, as for the norm test.
+    """
+    if not (theta > 0.0 and math.isfinite(theta) and nu > 0.0 and math.isfinite(nu)):
+        raise ValueError("theta and nu must be positive and finite")
+    G = np.asarray(G)
+    b, P = G.shape
+    total = np.zeros(P, dtype=np.float64)
+    for i in range(b):
+        total += widen(G[i])
+    gbar = total / b
+    N = float(np.dot(gbar, gbar))
+    r = InnerProductResult(mean_sqnorm=N, batch_count=b)
+    if b - ddof <= 0:
+        r.flags |= FLAG_UNDEFINED
+        r.b_ip = r.b_aug = max(1, b_cur)
+    elif N == 0.0:
+        r.flags |= FLAG_ZERO_MEAN
+        r.stat_ip = r.stat_orth = math.inf
+        r.b_ip = r.b_aug = b_cap if b_cap > 0 else INT64_MAX
+    else:
+        p = np.zeros(b, dtype=np.float64)
+        for i in range(b):
+            p[i] = float(np.dot(widen(G[i]), gbar))
+        pbar = float(p.sum()) / b
+        r.var_ip = float(((p - pbar) ** 2).sum()) / (b - ddof)
+        r.stat_ip = r.var_ip / (theta * theta * N * N)
+        obar = np.zeros(P, dtype=np.float64)
+        for i in range(b):
+            obar += widen(G[i]) - (p[i] / N) * gbar
+        obar /= b
+        dev = 0.0
+        for i in range(b):
+            c = widen(G[i]) - (p[i] / N) * gbar - obar
+            dev += float(np.dot(c, c))
+        r.var_orth = dev / (b - ddof)
+        r.stat_orth = r.var_orth / (nu * nu * N)
+        r.b_ip = max(1, math.ceil(r.stat_ip)) if r.stat_ip < 9.0e18 else INT64_MAX
+        b_orth = max(1, math.ceil(r.stat_orth)) if r.stat_orth < 9.0e18 else INT64_MAX
+        r.b_aug = max(r.b_ip, b_orth)
+        r.inner_products = p
+    if b_cap > 0:
+        r.b_ip, r.b_aug = min(r.b_ip, b_cap), min(r.b_aug, b_cap)
+    if r.b_aug > b_cur:
+        r.flags |= FLAG_GROW
+    return r
+
+
+# --------------------------------------------------------------------------
 # linear layers: per-sample weight gradients from activations and output grads
 # --------------------------------------------------------------------------
 def per_sample_weight_grad(X_i, D_i) -> np.ndarray:

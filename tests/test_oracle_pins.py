@@ -288,6 +288,60 @@ def pin_merge(O):
     assert np.array_equal(x, np.array([2.0, 0.0])) and rep == 0
 
 
+def exact_inner_product_tests(G, theta, nu, ddof):
+    """The two inner-product statistics in exact rationals, from their definitions."""
+    b, P = len(G), len(G[0])
+    g = [[Fraction(x) for x in row] for row in G]
+    gbar = [sum(g[i][j] for i in range(b)) / b for j in range(P)]
+    N = sum(x * x for x in gbar)
+    p = [sum(g[i][j] * gbar[j] for j in range(P)) for i in range(b)]
+    pbar = sum(p) / b
+    var_ip = sum((x - pbar) ** 2 for x in p) / (b - ddof)
+    o = [[g[i][j] - p[i] / N * gbar[j] for j in range(P)] for i in range(b)]
+    obar = [sum(o[i][j] for i in range(b)) / b for j in range(P)]
+    var_o = sum((o[i][j] - obar[j]) ** 2 for i in range(b) for j in range(P)) / (b - ddof)
+    return var_ip / (Fraction(theta) ** 2 * N * N), var_o / (Fraction(nu) ** 2 * N)
+
+
+def pin_inner_product_tests(O):
+    rng = np.random.default_rng(17)
+    for b, P, theta, nu, ddof in [(3, 4, 0.5, 0.25, 1), (5, 6, 0.125, 0.5, 1), (4, 3, 2.0, 1.0, 0)]:
+        G = int_matrix(rng, b, P)
+        G[:, 0] += 3.0      # keep the mean away from zero
+        s_ip, s_or = exact_inner_product_tests(G.tolist(), theta, nu, ddof)
+        r = O.inner_product_tests(G, theta=theta, nu=nu, ddof=ddof, b_cur=1)
+        assert math.isclose(r.stat_ip, float(s_ip), rel_tol=1e-12)
+        assert math.isclose(r.stat_orth, float(s_or), rel_tol=1e-12)
+        assert r.b_ip == max(1, math.ceil(s_ip))
+        assert r.b_aug == max(r.b_ip, max(1, math.ceil(s_or)))
+    # orthonormal gradients: every <g_i, gbar> equals ||gbar||^2, so the inner-product
+    # statistic vanishes; the orthogonal parts e_i - gbar give variance 1 and b / nu^2
+    G = np.eye(16, dtype=np.float32)[:8]
+    r = O.inner_product_tests(G, theta=0.01, nu=0.5, b_cur=1)
+    assert r.stat_ip < 1e-25 and r.b_ip == 1
+    assert math.isclose(r.var_orth, 1.0, rel_tol=1e-14) and math.isclose(r.stat_orth, 32.0, rel_tol=1e-14)
+    assert r.b_aug == 32 and r.flags & O.FLAG_GROW
+    # collinear gradients g_i = a_i u: no orthogonal part; stat_ip = Var(a) / (theta^2 abar^2)
+    a = np.array([1.0, 2.0, 3.0, 6.0])
+    u = np.zeros(8); u[2] = 1.0
+    G = (a[:, None] * u[None, :]).astype(np.float32)
+    r = O.inner_product_tests(G, theta=0.5, nu=0.3, b_cur=1)
+    assert r.var_orth < 1e-25 and math.isclose(r.stat_ip, a.var(ddof=1) / (0.25 * a.mean() ** 2), rel_tol=1e-14)
+    assert r.b_aug == r.b_ip == math.ceil(a.var(ddof=1) / (0.25 * 9.0))
+    # scale invariance of both statistics, caps, degenerate cases
+    G = W.to_numpy(W.per_sample_grads(6, 300, sigma=0.5, seed=4))
+    x = O.inner_product_tests(G, theta=0.1, nu=0.3)
+    y = O.inner_product_tests(G * np.float32(8.0), theta=0.1, nu=0.3)
+    assert math.isclose(x.stat_ip, y.stat_ip, rel_tol=1e-12) and math.isclose(x.stat_orth, y.stat_orth, rel_tol=1e-12)
+    assert O.inner_product_tests(G, theta=0.1, nu=0.3, b_cap=3).b_aug == 3
+    z = O.inner_product_tests(G[:1], theta=0.1, nu=0.3, b_cur=5)
+    assert z.flags & O.FLAG_UNDEFINED and z.b_ip == z.b_aug == 5
+    zero = np.array([[1.0, -1.0], [-1.0, 1.0]], dtype=np.float32)
+    assert O.inner_product_tests(zero, theta=0.1, nu=0.3).flags & O.FLAG_ZERO_MEAN
+    with pytest.raises(ValueError):
+        O.inner_product_tests(G, theta=0.0, nu=0.3)
+
+
 PINS = [v for k, v in sorted(globals().items()) if k.startswith("pin_")]
 
 
@@ -323,6 +377,12 @@ MUTANTS = [
     ("merge takes the largest", "order = sorted(range(k), key=lambda i: (b_req[i], i))",
      "order = sorted(range(k), key=lambda i: (-b_req[i], i))"),
     ("merge unweighted", "x += float(b) * widen(p)", "x += widen(p)"),
+    ("inner products against the sum", "p[i] = float(np.dot(widen(G[i]), gbar))", "p[i] = float(np.dot(widen(G[i]), total))"),
+    ("inner-product statistic with ||gbar||^2 only", "r.var_ip / (theta * theta * N * N)", "r.var_ip / (theta * theta * N)"),
+    ("projection not normalised", "c = widen(G[i]) - (p[i] / N) * gbar - obar", "c = widen(G[i]) - p[i] * gbar - obar"),
+    ("orthogonal statistic with theta", "r.var_orth / (nu * nu * N)", "r.var_orth / (theta * theta * N)"),
+    ("augmented test takes the min", "r.b_aug = max(r.b_ip, b_orth)", "r.b_aug = min(r.b_ip, b_orth)"),
+    ("inner-product variance uncentred", "float(((p - pbar) ** 2).sum()) / (b - ddof)", "float((p ** 2).sum()) / (b - ddof)"),
 ]
 
 
