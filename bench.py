@@ -488,7 +488,14 @@ def run_table(args):
     Gn = W.to_numpy(G)
     emit(2, "norm_test + eta sweep (B=64, P=2^24)", ms, nbytes=4 * 64 * (1 << 24),
          oracle_s=cpu_s(lambda: O.norm_test(Gn, eta=0.1)), oracle_note="whole")
-    del G, Gn
+    Ssum = torch.empty(1 << 24, device=dev)
+    ctx.norm_test(G, p, grad_sum=Ssum, sync=False)
+    ms = gpu_ms(lambda: ctx.inner_product_test(G, Ssum, theta=0.01, nu=0.3, b_cur=64), reps=10)
+    Gs = Gn[:, : 1 << 21]
+    o_s = cpu_s(lambda: O.inner_product_tests(Gs, theta=0.01, nu=0.3)) * 8
+    emit(2, "inner_product_test (second pass, B=64, P=2^24)", ms, nbytes=4 * 64 * (1 << 24) + 4 * (1 << 24),
+         oracle_s=o_s, oracle_note="timed on P=2^21, extrapolated", note="includes the host synchronisation of the call")
+    del G, Gn, Gs, Ssum
     outer_case(2, 8, W.GPT2_SMALL_P, torch.bfloat16)
     # config 3
     X, D = W.linear_layer(GR_B, GR_T, GR_DIN, GR_DOUT, seed=3, device=dev)

@@ -181,6 +181,48 @@ int adloco_norm_test_noalloc(const float* grads, int64_t B, int64_t P, int64_t r
                              const adloco_test_params* params, float* per_sample_sqnorm,
                              adloco_test_result* result_dev, adloco_test_result* result_host, void* stream);
 
+/* ---- inner-product test and augmented inner-product test ------------------ */
+
+/* Parameters: theta and nu are the thresholds of the two tests (> 0, finite);
+ * ddof, b_cur, b_cap as in adloco_test_params. */
+typedef struct {
+    double theta;
+    double nu;
+    int32_t ddof;
+    int32_t reserved;
+    int64_t b_cur;
+    int64_t b_cap;
+} adloco_ip_params;
+
+/* var_ip = Var_i <g_i, gbar>, stat_ip = var_ip / (theta^2 ||gbar||^4), b_ip = max(1, ceil(stat_ip));
+ * var_orth = Var_i (g_i - (<g_i, gbar> / ||gbar||^2) gbar), stat_orth = var_orth / (nu^2 ||gbar||^2),
+ * b_aug = max(b_ip, ceil(stat_orth)).  Flags GROW (b_aug > b_cur), UNDEFINED, ZERO_MEAN as for the norm test. */
+typedef struct {
+    double var_ip;
+    double stat_ip;
+    double var_orth;
+    double stat_orth;
+    double mean_sqnorm;
+    int64_t batch_count;
+    int64_t b_ip;
+    int64_t b_aug;
+    uint32_t flags;
+    int32_t device_status;
+} adloco_ip_result;
+
+/* Section "Inner product test": both batch rules for the batch whose norm test
+ * has just run.  A second pass over G:
+ *   grads, B, P, row_stride   as in adloco_norm_test (the same G)
+ *   grad_sum                  dev [P] float: S = sum_i g_i, the grad_sum output of that norm test (required)
+ *   sums_dev                  dev: the sums_dev output of that norm test (required)
+ *   inner_products            dev [B] float, receives <g_i, gbar>; may be NULL
+ *   result_dev / result_host  as in adloco_norm_test
+ * Algorithmic traffic 4 B P + 4 P bytes. */
+int adloco_inner_product_test(adloco_ctx* ctx, const void* grads, adloco_dtype dtype, int64_t B, int64_t P,
+                              int64_t row_stride, const adloco_ip_params* params, const float* grad_sum,
+                              const adloco_test_sums* sums_dev, float* inner_products,
+                              adloco_ip_result* result_dev, adloco_ip_result* result_host, void* stream);
+
 /* ---- per-sample norms of a linear layer via the Gram identity ------------ */
 
 /* For a linear layer y = W x and a batch of B sequences of T tokens, sample i

@@ -23,7 +23,7 @@ FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN = 1, 2, 4, 8
 EXPORTS = (
     "adloco_create", "adloco_destroy", "adloco_status_string", "adloco_last_cuda_error", "adloco_launch_count",
     "adloco_set_wait_limit", "adloco_device_status",
-    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_gram_sqnorm", "adloco_linear_sqnorm",
+    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_inner_product_test", "adloco_gram_sqnorm", "adloco_linear_sqnorm",
     "adloco_accum_create", "adloco_accum_reset", "adloco_accum_destroy", "adloco_accumulate",
     "adloco_accum_finalize", "adloco_outer_step", "adloco_outer_step_host", "adloco_check_merge", "adloco_merge",
 )
@@ -50,6 +50,17 @@ class TestResult(C.Structure):
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class IpParams(C.Structure):
+    _fields_ = [("theta", C.c_double), ("nu", C.c_double), ("ddof", C.c_int32), ("reserved", C.c_int32),
+                ("b_cur", C.c_int64), ("b_cap", C.c_int64)]
+
+
+class IpResult(C.Structure):
+    _fields_ = [("var_ip", C.c_double), ("stat_ip", C.c_double), ("var_orth", C.c_double),
+                ("stat_orth", C.c_double), ("mean_sqnorm", C.c_double), ("batch_count", C.c_int64),
+                ("b_ip", C.c_int64), ("b_aug", C.c_int64), ("flags", C.c_uint32), ("device_status", C.c_int32)]
 
 
 class AdlocoError(RuntimeError):
@@ -82,6 +93,7 @@ def load_library() -> C.CDLL:
         "adloco_test_decide": (C.c_int, [vp, vp, C.POINTER(TestParams), vp, vp, vp]),
         "adloco_norm_test_host": (C.c_int, [vp, vp, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp]),
         "adloco_norm_test_noalloc": (C.c_int, [vp, i64, i64, i64, C.POINTER(TestParams), vp, vp, vp, vp]),
+        "adloco_inner_product_test": (C.c_int, [vp, vp, C.c_int, i64, i64, i64, C.POINTER(IpParams), vp, vp, vp, vp, vp, vp]),
         "adloco_gram_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
         "adloco_linear_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, C.c_int, vp]),
         "adloco_accum_create": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), i32]),
@@ -211,6 +223,23 @@ class Context:
                                             C.cast(C.byref(res), C.c_void_p), _stream(stream))
         self.check(rc, "adloco_norm_test_host")
         return res
+
+    def inner_product_test(self, G, grad_sum, *, theta, nu, ddof=1, b_cur=1, b_cap=0, inner_products=None,
+                           sums_dev=None, stream=None) -> IpResult:
+        """adloco_inner_product_test on the G whose norm test (with grad_sum) has just run on this context."""
+        B, P = G.shape
+        stride = G.stride(0) if B > 1 else max(G.stride(0), P)
+        p = IpParams(float(theta), float(nu), int(ddof), 0, int(b_cur), int(b_cap))
+        if not hasattr(self, "_ip_dev"):
+            self._ip_dev = torch.zeros(C.sizeof(IpResult), dtype=torch.uint8, device=self.device)
+            self._ip_host = torch.zeros(C.sizeof(IpResult), dtype=torch.uint8).pin_memory()
+        s = self._sums_dev if sums_dev is None else sums_dev
+        rc = self.lib.adloco_inner_product_test(self.h, _ptr(G), _dtype_code(G.dtype), B, P, stride, C.byref(p),
+                                                _ptr(grad_sum), _ptr(s), _ptr(inner_products), _ptr(self._ip_dev),
+                                                _ptr(self._ip_host), _stream(stream))
+        self.check(rc, "adloco_inner_product_test")
+        (stream or torch.cuda.current_stream()).synchronize()
+        return IpResult.from_buffer_copy(self._ip_host.numpy().tobytes())
 
     # ------------------------------------------------------------------ Gram path
     def gram_sqnorm(self, X, D, per_sample_sqnorm, *, accumulate_norms=False, grad_sum=None,

@@ -239,6 +239,30 @@ int adloco_norm_test_host(adloco_ctx* ctx, const float* grads_host, int64_t B, i
     return ADLOCO_OK;
 }
 
+int adloco_inner_product_test(adloco_ctx* ctx, const void* grads, adloco_dtype dtype, int64_t B, int64_t P,
+                              int64_t row_stride, const adloco_ip_params* params, const float* grad_sum,
+                              const adloco_test_sums* sums_dev, float* inner_products,
+                              adloco_ip_result* result_dev, adloco_ip_result* result_host, void* stream) {
+    if (!ctx || !params || !grad_sum || !sums_dev || !result_dev) return ADLOCO_ERR_INVALID_ARG;
+    if (!(params->theta > 0.0) || !(params->theta < 1.0e300) || !(params->nu > 0.0) || !(params->nu < 1.0e300))
+        return ADLOCO_ERR_INVALID_ARG;
+    if (params->ddof < 0 || params->b_cur < 0 || params->b_cap < 0) return ADLOCO_ERR_INVALID_ARG;
+    int rc = check_grads(grads, dtype, B, P, row_stride);
+    if (rc != ADLOCO_OK) return rc;
+    if ((reinterpret_cast<uintptr_t>(grad_sum) & 3u) != 0) return ADLOCO_ERR_ALIGNMENT;
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    IpLaunch l;
+    l.G = static_cast<const float*>(grads);
+    l.S = grad_sum; l.B = B; l.P = P; l.stride = row_stride; l.sums = sums_dev; l.params = *params;
+    l.dots_out = inner_products; l.result = result_dev;
+    rc = launch_inner_product(ctx, l, st);
+    if (rc != ADLOCO_OK) return rc;
+    if (result_host)
+        ADLOCO_CUDA_TRY(ctx, cudaMemcpyAsync(result_host, result_dev, sizeof(adloco_ip_result), cudaMemcpyDeviceToHost, st));
+    return ADLOCO_OK;
+}
+
 // ---------------------------------------------------------------------------------
 // Gram path
 // ---------------------------------------------------------------------------------

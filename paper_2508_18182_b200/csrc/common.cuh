@@ -107,6 +107,17 @@ int launch_norm_test(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st);
 int launch_decide(adloco_ctx* ctx, const adloco_test_sums* sums, const adloco_test_params& p,
                   adloco_test_result* result, cudaStream_t st);
 
+struct IpLaunch {
+    const float* G = nullptr;
+    const float* S = nullptr;
+    int64_t B = 0, P = 0, stride = 0;
+    const adloco_test_sums* sums = nullptr;
+    adloco_ip_params params{};
+    float* dots_out = nullptr;
+    adloco_ip_result* result = nullptr;
+};
+int launch_inner_product(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st);
+
 struct OuterLaunch {
     const void* inst[kMaxInstances];
     void* wb[kMaxInstances];

@@ -409,6 +409,207 @@ int launch_decide(adloco_ctx* ctx, const adloco_test_sums* sums, const adloco_te
 }
 
 // ---------------------------------------------------------------------------------
+// inner-product tests: second pass over G with the gradient sum S of the first
+// ---------------------------------------------------------------------------------
+struct IpArgs {
+    const float* G;
+    const float* S;            // [P] sum of the rows of G (adloco_norm_test's grad_sum)
+    int64_t B, P, stride;
+    const adloco_test_sums* sums;   // of the norm test on the same G
+    adloco_ip_params params;
+    float* dots_out;           // [B] <g_i, gbar>, may be null
+    adloco_ip_result* result;
+    float* n_partials;
+    unsigned* ticket;
+    int iters;
+};
+
+// Batch rules of the inner-product test and its augmented form from
+//   d_i = <g_i, gbar> - ||gbar||^2 (i = 0..b-1, their sum of squares and mean given),
+//   css = sum_i ||g_i - gbar||^2,  N = ||gbar||^2:
+//   Var_i <g_i, gbar> = sum (d_i - dbar)^2 / (b - ddof)
+//   the parts of the g_i orthogonal to gbar have mean zero and
+//   sum_i ||o_i||^2 = css - sum_i d_i^2 / N.
+__device__ void ip_decide_device(double sum_d2, double sum_d, const adloco_test_sums& s, const adloco_ip_params& p,
+                                 adloco_ip_result* out) {
+    adloco_ip_result r;
+    const int64_t b = s.batch_count;
+    const double bd = (double)b;
+    const double N = b > 0 ? s.sum_sq_gsum / (bd * bd) : 0.0;
+    const int64_t i64max = 0x7fffffffffffffffLL;
+    r.mean_sqnorm = N;
+    r.batch_count = b;
+    r.flags = 0;
+    r.device_status = s.device_status;
+    r.var_ip = r.stat_ip = r.var_orth = r.stat_orth = 0.0;
+    if (b - p.ddof <= 0) {
+        r.flags |= ADLOCO_FLAG_UNDEFINED;
+        r.b_ip = r.b_aug = p.b_cur > 1 ? p.b_cur : 1;
+    } else if (N == 0.0) {
+        r.flags |= ADLOCO_FLAG_ZERO_MEAN;
+        r.stat_ip = r.stat_orth = __longlong_as_double(0x7ff0000000000000LL);
+        r.b_ip = r.b_aug = p.b_cap > 0 ? p.b_cap : i64max;
+    } else {
+        const double denom = (double)(b - p.ddof);
+        double centred = sum_d2 - sum_d * sum_d / bd;
+        if (centred < 0.0) centred = 0.0;
+        r.var_ip = centred / denom;
+        r.stat_ip = r.var_ip / (p.theta * p.theta * N * N);
+        const double css = s.has_centred ? s.centred_ss : s.sum_sqnorm - bd * N;
+        double orth = css - sum_d2 / N;
+        if (orth < 0.0) orth = 0.0;
+        r.var_orth = orth / denom;
+        r.stat_orth = r.var_orth / (p.nu * p.nu * N);
+        const int64_t c_ip = r.stat_ip < 9.0e18 ? (int64_t)ceil(r.stat_ip) : i64max;
+        const int64_t c_or = r.stat_orth < 9.0e18 ? (int64_t)ceil(r.stat_orth) : i64max;
+        r.b_ip = c_ip > 1 ? c_ip : 1;
+        r.b_aug = c_or > r.b_ip ? c_or : r.b_ip;
+    }
+    if (p.b_cap > 0) {
+        if (r.b_ip > p.b_cap) r.b_ip = p.b_cap;
+        if (r.b_aug > p.b_cap) r.b_aug = p.b_cap;
+    }
+    if (r.b_aug > p.b_cur) r.flags |= ADLOCO_FLAG_GROW;
+    *out = r;
+}
+
+// Thread layout as in norm_test_kernel: a thread owns four adjacent columns, loads
+// their entries of S once and walks down the rows accumulating, per row,
+// sum_j (G_ij - S_j / b) S_j = b (<g_i, gbar> - ||gbar||^2): centring before the
+// product keeps the small deviation d_i free of cancellation.
+template <int RB, bool VEC>
+__global__ void __launch_bounds__(NT_THREADS, 2) centred_dot_kernel(const __grid_constant__ IpArgs a) {
+    extern __shared__ float smem_rows[];  // [NT_WARPS][Bpad]
+    __shared__ double smem_red[32];
+    __shared__ int smem_is_last;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t B = a.B;
+    const int Bpad = (int)(((B + RB - 1) / RB) * RB);
+    for (int i = tid; i < NT_WARPS * Bpad; i += NT_THREADS) smem_rows[i] = 0.f;
+    __syncthreads();
+    float* my_rows = smem_rows + warp * Bpad;
+    const int64_t ngroups = (a.P + 3) >> 2;
+    const bool single_tile = (B <= RB);
+    const float invB = 1.0f / (float)B;
+
+    float acc[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) acc[r] = 0.f;
+
+    for (int it = 0; it < a.iters; ++it) {
+        const int64_t g = ((int64_t)it * gridDim.x + blockIdx.x) * NT_THREADS + tid;
+        const int64_t col = g << 2;
+        int nvalid = 0;
+        if (g < ngroups) nvalid = (a.P - col) >= 4 ? 4 : (int)(a.P - col);
+        const float* rowp = a.G + (nvalid > 0 ? col : 0);
+        const float4 s4 = load4<VEC>(a.S + (nvalid > 0 ? col : 0), nvalid);
+        const float4 m4 = make_float4(s4.x * invB, s4.y * invB, s4.z * invB, s4.w * invB);
+        for (int64_t i0 = 0; i0 < B; i0 += RB) {
+#pragma unroll
+            for (int r0 = 0; r0 < RB; r0 += NT_CHUNK) {
+                float4 x[NT_CHUNK];
+#pragma unroll
+                for (int u = 0; u < NT_CHUNK; ++u) {
+                    const bool ok = (i0 + r0 + u) < B;
+                    x[u] = load4<VEC>(rowp + (int64_t)(r0 + u) * a.stride, ok ? nvalid : 0);
+                }
+#pragma unroll
+                for (int u = 0; u < NT_CHUNK; ++u) {
+                    if ((i0 + r0 + u) < B) {
+                        // columns beyond P carry s4 = 0 and add nothing
+                        float q = (x[u].x - m4.x) * s4.x;
+                        q = fmaf(x[u].y - m4.y, s4.y, q);
+                        q = fmaf(x[u].z - m4.z, s4.z, q);
+                        q = fmaf(x[u].w - m4.w, s4.w, q);
+                        acc[r0 + u] += q;
+                    }
+                }
+            }
+            rowp += (int64_t)RB * a.stride;
+            if (!single_tile) {
+                warp_rows_flush<RB>(acc, my_rows + i0, lane);
+#pragma unroll
+                for (int r = 0; r < RB; ++r) acc[r] = 0.f;
+            }
+        }
+    }
+    if (single_tile) warp_rows_flush<RB>(acc, my_rows, lane);
+    __syncthreads();
+    for (int64_t i = tid; i < B; i += NT_THREADS) {
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < NT_WARPS; ++w) t += smem_rows[w * Bpad + i];
+        a.n_partials[(int64_t)blockIdx.x * B + i] = t;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) smem_is_last = (atomicAdd(a.ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!smem_is_last) return;
+    __threadfence();
+
+    // last block: d_i in fp64, fixed order
+    const adloco_test_sums s = *a.sums;
+    const double bd = (double)B;
+    const double N = s.sum_sq_gsum / (bd * bd);
+    double l_d2 = 0.0, l_d = 0.0;
+    for (int64_t i = tid; i < B; i += NT_THREADS) {
+        double t = 0.0;
+        for (unsigned blk = 0; blk < gridDim.x; ++blk) t += (double)__ldcg(a.n_partials + (int64_t)blk * B + i);
+        const double d = t / bd;
+        if (a.dots_out != nullptr) a.dots_out[i] = (float)(N + d);
+        l_d2 += d * d;
+        l_d += d;
+    }
+    const double sum_d2 = block_sum(l_d2, smem_red);
+    const double sum_d = block_sum(l_d, smem_red);
+    if (tid == 0) {
+        ip_decide_device(sum_d2, sum_d, s, a.params, a.result);
+        *a.ticket = 0u;
+    }
+}
+
+template <int RB, bool VEC>
+static int launch_ip_t(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
+    const int64_t ngroups = (l.P + 3) / 4;
+    const int64_t tiles = (ngroups + NT_THREADS - 1) / NT_THREADS;
+    const int Bpad = (int)(((l.B + RB - 1) / RB) * RB);
+    const size_t smem = (size_t)NT_WARPS * Bpad * sizeof(float);
+    auto kern = centred_dot_kernel<RB, VEC>;
+    if (smem > 48 * 1024) ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NT_THREADS, smem));
+    if (per_sm < 1) return ADLOCO_ERR_WORKSPACE;
+    int64_t max_grid = (int64_t)ctx->sm_count * per_sm;
+    if (max_grid > ctx->max_grid) max_grid = ctx->max_grid;
+    const int64_t iters = (tiles + max_grid - 1) / max_grid;
+    const int64_t grid = (tiles + iters - 1) / iters;
+    int rc = grow_workspace(ctx, (size_t)grid * (size_t)l.B);
+    if (rc != ADLOCO_OK) return rc;
+    IpArgs a;
+    a.G = l.G; a.S = l.S; a.B = l.B; a.P = l.P; a.stride = l.stride; a.sums = l.sums; a.params = l.params;
+    a.dots_out = l.dots_out; a.result = l.result;
+    a.n_partials = ctx->n_partials; a.ticket = ctx->ticket; a.iters = (int)iters;
+    kern<<<(unsigned)grid, NT_THREADS, smem, st>>>(a);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+int launch_inner_product(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
+    const bool vec = aligned16(l.G) && aligned16(l.S) && (l.B == 1 || (l.stride % 4) == 0);
+    if (vec) {
+        if (l.B <= 16) return launch_ip_t<16, true>(ctx, l, st);
+        if (l.B <= 32) return launch_ip_t<32, true>(ctx, l, st);
+        return launch_ip_t<64, true>(ctx, l, st);
+    }
+    if (l.B <= 16) return launch_ip_t<16, false>(ctx, l, st);
+    if (l.B <= 32) return launch_ip_t<32, false>(ctx, l, st);
+    return launch_ip_t<64, false>(ctx, l, st);
+}
+
+// ---------------------------------------------------------------------------------
 // norm test without any allocation
 // ---------------------------------------------------------------------------------
 // Some callers cannot allocate device memory at the point where they need the
