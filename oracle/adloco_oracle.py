@@ -258,6 +258,22 @@ def linear_layer_terms(X, D):
     return n, S
 
 
+def vector_param_terms(D, X=None):
+    """Per-sample gradients of a vector parameter of width d applied at every token:
+    a bias (y_t = ... + beta: g_i = sum_t delta_t) or an elementwise gain such as
+    LayerNorm's (y_t = gamma * xhat_t: g_i = sum_t delta_t * xhat_t, X = xhat).
+    D [B, T, d] (and X [B, T, d]).  Returns n_i = ||g_i||^2 and S = sum_i g_i."""
+    B = D.shape[0]
+    n = np.zeros(B, dtype=np.float64)
+    S = np.zeros(D.shape[2], dtype=np.float64)
+    for i in range(B):
+        d = widen(D[i])
+        g = (d * widen(X[i])).sum(axis=0) if X is not None else d.sum(axis=0)
+        n[i] = float(np.dot(g, g))
+        S += g
+    return n, S
+
+
 def linear_layers_norm_test(layers, *, eta: float, ddof: int = 1, b_cur: int = 1,
                             b_max: int = 1, b_cap: int = 0, switch_n: int = 2,
                             two_pass: bool = True) -> NormTestResult:

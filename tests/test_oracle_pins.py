@@ -203,6 +203,25 @@ def pin_linear_layer_brute_force(O):
         assert n1[i] == float((X1[i].float() ** 2).sum() * (D1[i].float() ** 2).sum())
 
 
+def pin_vector_param_terms(O):
+    X, D = W.small_integer_layer(3, 5, 6, 6, seed=13)
+    Xi, Di = X.float().numpy(), D.float().numpy()
+    n, S = O.vector_param_terms(W.to_numpy(D))
+    n2, S2 = O.vector_param_terms(W.to_numpy(D), W.to_numpy(X))
+    S_ref, S2_ref = [0] * 6, [0] * 6
+    for i in range(3):
+        g = [sum(int(Di[i][t][j]) for t in range(5)) for j in range(6)]
+        g2 = [sum(int(Di[i][t][j]) * int(Xi[i][t][j]) for t in range(5)) for j in range(6)]
+        assert n[i] == float(sum(x * x for x in g)) and n2[i] == float(sum(x * x for x in g2))
+        S_ref = [a + c for a, c in zip(S_ref, g)]
+        S2_ref = [a + c for a, c in zip(S2_ref, g2)]
+    assert S.tolist() == [float(x) for x in S_ref] and S2.tolist() == [float(x) for x in S2_ref]
+    # a bias is the weight of a constant input 1: same norms as the linear layer with X = ones [T, 1]
+    ones = torch.ones(3, 5, 1, dtype=torch.bfloat16)
+    n_lin, S_lin = O.linear_layer_terms(W.to_numpy(ones), W.to_numpy(D))
+    assert np.array_equal(n_lin, n) and np.array_equal(S_lin[:, 0], S)
+
+
 def pin_layers_test_two_routes(O):
     layers = [tuple(W.to_numpy(t) for t in W.linear_layer(4, 6, 8, 16, seed=1)),
               tuple(W.to_numpy(t) for t in W.linear_layer(4, 6, 16, 8, seed=2))]
@@ -377,6 +396,10 @@ MUTANTS = [
     ("merge takes the largest", "order = sorted(range(k), key=lambda i: (b_req[i], i))",
      "order = sorted(range(k), key=lambda i: (-b_req[i], i))"),
     ("merge unweighted", "x += float(b) * widen(p)", "x += widen(p)"),
+    ("vector parameter summed over features", "g = (d * widen(X[i])).sum(axis=0) if X is not None else d.sum(axis=0)",
+     "g = (d * widen(X[i])).sum(axis=1) if X is not None else d.sum(axis=1)"),
+    ("gain gradient without the input", "g = (d * widen(X[i])).sum(axis=0) if X is not None else d.sum(axis=0)",
+     "g = d.sum(axis=0)"),
     ("inner products against the sum", "p[i] = float(np.dot(widen(G[i]), gbar))", "p[i] = float(np.dot(widen(G[i]), total))"),
     ("inner-product statistic with ||gbar||^2 only", "r.var_ip / (theta * theta * N * N)", "r.var_ip / (theta * theta * N)"),
     ("projection not normalised", "c = widen(G[i]) - (p[i] / N) * gbar - obar", "c = widen(G[i]) - p[i] * gbar - obar"),
