@@ -512,6 +512,11 @@ def run_table(args):
     emit(3, "mean-gradient GEMM (difference)", ms_gs - ms_g, flops=mg)
     emit(3, "linear_sqnorm direct (norms + gradient sum)", ms_d, flops=mg, oracle_s=o_s, oracle_note="whole",
          note="same outputs as the row above from one GEMM")
+    Sb = torch.zeros(GR_DOUT, device=dev)
+    ms_b = gpu_ms(lambda: ctx.vector_param_sqnorm(D, n, grad_sum=Sb), flush=True)
+    Dn8 = Dn[:8]
+    emit(3, "vector_param_sqnorm (bias of the layer, Delta [32,1024,3072])", ms_b, nbytes=2 * GR_B * GR_T * GR_DOUT,
+         oracle_s=cpu_s(lambda: O.vector_param_terms(Dn8)) * 4, oracle_note="8 samples timed, x4", note="L2 flushed")
     # config 4: 12 blocks x 4 layers x 4 micro-batches, all inputs resident (38.7 GB)
     shapes = list(W.GPT2_SMALL_BLOCK_LINEARS) * 12
     data = [[W.linear_layer(32, 1024, di, do, seed=1000 * j + l, device=dev) for l, (di, do) in enumerate(shapes)]

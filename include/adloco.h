@@ -255,6 +255,18 @@ int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
                          int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
                          int accumulate_sum, int method, void* stream);
 
+/* Per-sample gradient norms of a vector parameter of width d that acts at every
+ * token (Eq. 1 applied to that parameter): a bias, g_i = sum_t delta_{i,t} (X = NULL),
+ * or an elementwise gain such as LayerNorm's, g_i = sum_t delta_{i,t} * x_{i,t}
+ * (X = the normalised input).  n_i = ||g_i||^2 and, optionally, S = sum_i g_i.
+ *   D, X               dev bf16 [B, T, d] row-major; d a multiple of 8, B <= 65535
+ *   per_sample_sqnorm  dev [B] float; overwritten, or += when accumulate_norms != 0
+ *   grad_sum           dev [d] float, may be NULL; overwritten, or += when accumulate_sum != 0
+ * One streaming pass (2 B T d bytes per operand), fp32 accumulation. */
+int adloco_vector_param_sqnorm(adloco_ctx* ctx, const void* D, const void* X, int64_t B, int64_t T, int64_t d,
+                               float* per_sample_sqnorm, int accumulate_norms, float* grad_sum, int accumulate_sum,
+                               void* stream);
+
 /* ---- switch-mode accumulation -------------------------------------------- */
 
 /* Accumulator of the test sums over the micro-batches of one large batch:

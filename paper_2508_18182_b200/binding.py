@@ -23,7 +23,7 @@ FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN = 1, 2, 4, 8
 EXPORTS = (
     "adloco_create", "adloco_destroy", "adloco_status_string", "adloco_last_cuda_error", "adloco_launch_count",
     "adloco_set_wait_limit", "adloco_device_status",
-    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_inner_product_test", "adloco_gram_sqnorm", "adloco_linear_sqnorm",
+    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_inner_product_test", "adloco_gram_sqnorm", "adloco_linear_sqnorm", "adloco_vector_param_sqnorm",
     "adloco_accum_create", "adloco_accum_reset", "adloco_accum_destroy", "adloco_accumulate",
     "adloco_accum_finalize", "adloco_outer_step", "adloco_outer_step_host", "adloco_check_merge", "adloco_merge",
 )
@@ -96,6 +96,7 @@ def load_library() -> C.CDLL:
         "adloco_inner_product_test": (C.c_int, [vp, vp, C.c_int, i64, i64, i64, C.POINTER(IpParams), vp, vp, vp, vp, vp, vp]),
         "adloco_gram_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
         "adloco_linear_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, C.c_int, vp]),
+        "adloco_vector_param_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
         "adloco_accum_create": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), i32]),
         "adloco_accum_reset": (C.c_int, [vp, vp, vp]),
         "adloco_accum_destroy": (C.c_int, [vp]),
@@ -265,6 +266,17 @@ class Context:
                                            int(accumulate_norms), _ptr(grad_sum), int(accumulate_sum), code,
                                            _stream(stream))
         self.check(rc, "adloco_linear_sqnorm")
+
+    def vector_param_sqnorm(self, D, per_sample_sqnorm, *, X=None, accumulate_norms=False, grad_sum=None,
+                            accumulate_sum=False, stream=None):
+        """adloco_vector_param_sqnorm: bias (X=None) or elementwise gain (X given)."""
+        B, T, d = D.shape
+        if D.dtype != torch.bfloat16 or not D.is_contiguous() or (X is not None and (X.shape != D.shape or not X.is_contiguous())):
+            raise AdlocoError(ERR_INVALID_ARG, "D (and X) must be contiguous bfloat16 of one shape")
+        rc = self.lib.adloco_vector_param_sqnorm(self.h, _ptr(D), _ptr(X), B, T, d, _ptr(per_sample_sqnorm),
+                                                 int(accumulate_norms), _ptr(grad_sum), int(accumulate_sum),
+                                                 _stream(stream))
+        self.check(rc, "adloco_vector_param_sqnorm")
 
     # ------------------------------------------------------------------ outer step
     def outer_step(self, instances, theta_in, mom_in, *, lr, momentum, nesterov=True, theta_out=None,

@@ -283,6 +283,18 @@ int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     return rc;
 }
 
+int adloco_vector_param_sqnorm(adloco_ctx* ctx, const void* D, const void* X, int64_t B, int64_t T, int64_t d,
+                               float* per_sample_sqnorm, int accumulate_norms, float* grad_sum, int accumulate_sum,
+                               void* stream) {
+    if (!ctx || !D || !per_sample_sqnorm) return ADLOCO_ERR_INVALID_ARG;
+    if (B < 1 || T < 1 || d < 1) return ADLOCO_ERR_INVALID_ARG;
+    if ((d % 8) != 0 || B > 65535) return ADLOCO_ERR_UNSUPPORTED;
+    if (!aligned16(D) || (X && !aligned16(X))) return ADLOCO_ERR_ALIGNMENT;
+    DeviceGuard g(ctx->device);
+    return launch_vec_param(ctx, D, X, B, T, d, per_sample_sqnorm, accumulate_norms, grad_sum, accumulate_sum,
+                            static_cast<cudaStream_t>(stream));
+}
+
 int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                          int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
                          int accumulate_sum, int method, void* stream) {

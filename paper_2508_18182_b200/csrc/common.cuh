@@ -118,6 +118,9 @@ struct IpLaunch {
 };
 int launch_inner_product(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st);
 
+int launch_vec_param(adloco_ctx* ctx, const void* D, const void* X, int64_t B, int64_t T, int64_t d, float* n,
+                     int accumulate_norms, float* S, int accumulate_sum, cudaStream_t st);
+
 struct OuterLaunch {
     const void* inst[kMaxInstances];
     void* wb[kMaxInstances];

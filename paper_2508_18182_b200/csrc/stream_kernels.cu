@@ -48,6 +48,10 @@ __device__ __forceinline__ void store4(float* p, float4 v, int nvalid) {
     }
 }
 
+// the two bfloat16 halves of a 32-bit word, widened exactly
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -610,6 +614,96 @@ int launch_inner_product(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
 }
 
 // ---------------------------------------------------------------------------------
+// vector parameters (bias, elementwise gain): g_i = sum_t delta_t (* x_t)
+// ---------------------------------------------------------------------------------
+struct VecParamArgs {
+    const __nv_bfloat16* D;
+    const __nv_bfloat16* X;   // null for a bias
+    int64_t T, d;
+    float* n;                 // [B], +=
+    float* S;                 // [d], += ; may be null
+};
+
+// Block (f, i) owns 256 adjacent features of sample i: a lane holds 8 of them (one
+// 128-bit load per token row), the 8 warps share the tokens; the per-warp sums meet in
+// shared memory, are squared into n_i and added into S.
+template <bool HAS_X>
+__global__ void __launch_bounds__(256) vec_param_kernel(const VecParamArgs a) {
+    __shared__ float part[8][257];
+    __shared__ double red[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t i = blockIdx.y;
+    const int64_t f0 = (int64_t)blockIdx.x * 256 + lane * 8;
+    const bool live = f0 < a.d;                      // d is a multiple of 8
+    const __nv_bfloat16* dp = a.D + (i * a.T) * a.d + f0;
+    const __nv_bfloat16* xp = HAS_X ? a.X + (i * a.T) * a.d + f0 : nullptr;
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    if (live) {
+        constexpr int U = 4;                         // token rows in flight per warp
+        for (int64_t t = warp; t < a.T; t += 8 * U) {
+            uint4 dv[U], xv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int64_t tt = t + (int64_t)u * 8;
+                dv[u] = make_uint4(0, 0, 0, 0);
+                xv[u] = make_uint4(0, 0, 0, 0);
+                if (tt < a.T) {
+                    dv[u] = __ldcs(reinterpret_cast<const uint4*>(dp + tt * a.d));
+                    if (HAS_X) xv[u] = __ldcs(reinterpret_cast<const uint4*>(xp + tt * a.d));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t dw[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+                const uint32_t xw[4] = {xv[u].x, xv[u].y, xv[u].z, xv[u].w};
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    if (HAS_X) {
+                        acc[2 * h] = fmaf(bf16_lo(dw[h]), bf16_lo(xw[h]), acc[2 * h]);
+                        acc[2 * h + 1] = fmaf(bf16_hi(dw[h]), bf16_hi(xw[h]), acc[2 * h + 1]);
+                    } else {
+                        acc[2 * h] += bf16_lo(dw[h]);
+                        acc[2 * h + 1] += bf16_hi(dw[h]);
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) part[warp][lane * 8 + e] = acc[e];
+    __syncthreads();
+    float g = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) g += part[w][threadIdx.x];
+    const int64_t f = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    double sq = 0.0;
+    if (f < a.d) {
+        sq = (double)g * (double)g;
+        if (a.S != nullptr) atomicAdd(a.S + f, g);
+    }
+    const double tot = block_sum(sq, red);
+    if (threadIdx.x == 0) atomicAdd(a.n + i, (float)tot);
+}
+
+int launch_vec_param(adloco_ctx* ctx, const void* D, const void* X, int64_t B, int64_t T, int64_t d, float* n,
+                     int accumulate_norms, float* S, int accumulate_sum, cudaStream_t st) {
+    if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
+    if (S && !accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d * sizeof(float), st));
+    VecParamArgs a;
+    a.D = static_cast<const __nv_bfloat16*>(D);
+    a.X = static_cast<const __nv_bfloat16*>(X);
+    a.T = T; a.d = d; a.n = n; a.S = S;
+    const dim3 grid((unsigned)((d + 255) / 256), (unsigned)B);
+    if (X) vec_param_kernel<true><<<grid, 256, 0, st>>>(a);
+    else vec_param_kernel<false><<<grid, 256, 0, st>>>(a);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+// ---------------------------------------------------------------------------------
 // norm test without any allocation
 // ---------------------------------------------------------------------------------
 // Some callers cannot allocate device memory at the point where they need the
@@ -731,8 +825,6 @@ struct OuterArgs {
     int K, nesterov;
 };
 
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&p);
