@@ -627,9 +627,12 @@ struct VecParamArgs {
 // Block (f, i) owns 256 adjacent features of sample i: a lane holds 8 of them (one
 // 128-bit load per token row), the 8 warps share the tokens; the per-warp sums meet in
 // shared memory, are squared into n_i and added into S.
+constexpr int VP_WARPS = 16;
+constexpr int VP_THREADS = 32 * VP_WARPS;
+
 template <bool HAS_X>
-__global__ void __launch_bounds__(256) vec_param_kernel(const VecParamArgs a) {
-    __shared__ float part[8][257];
+__global__ void __launch_bounds__(VP_THREADS) vec_param_kernel(const VecParamArgs a) {
+    __shared__ float part[VP_WARPS][257];
     __shared__ double red[32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t i = blockIdx.y;
@@ -641,12 +644,12 @@ __global__ void __launch_bounds__(256) vec_param_kernel(const VecParamArgs a) {
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
     if (live) {
-        constexpr int U = 4;                         // token rows in flight per warp
-        for (int64_t t = warp; t < a.T; t += 8 * U) {
+        constexpr int U = 8;                         // token rows in flight per warp
+        for (int64_t t = warp; t < a.T; t += VP_WARPS * U) {
             uint4 dv[U], xv[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int64_t tt = t + (int64_t)u * 8;
+                const int64_t tt = t + (int64_t)u * VP_WARPS;
                 dv[u] = make_uint4(0, 0, 0, 0);
                 xv[u] = make_uint4(0, 0, 0, 0);
                 if (tt < a.T) {
@@ -675,11 +678,13 @@ __global__ void __launch_bounds__(256) vec_param_kernel(const VecParamArgs a) {
     for (int e = 0; e < 8; ++e) part[warp][lane * 8 + e] = acc[e];
     __syncthreads();
     float g = 0.f;
+    if (threadIdx.x < 256) {
 #pragma unroll
-    for (int w = 0; w < 8; ++w) g += part[w][threadIdx.x];
+        for (int w = 0; w < VP_WARPS; ++w) g += part[w][threadIdx.x];
+    }
     const int64_t f = (int64_t)blockIdx.x * 256 + threadIdx.x;
     double sq = 0.0;
-    if (f < a.d) {
+    if (threadIdx.x < 256 && f < a.d) {
         sq = (double)g * (double)g;
         if (a.S != nullptr) atomicAdd(a.S + f, g);
     }
@@ -696,8 +701,8 @@ int launch_vec_param(adloco_ctx* ctx, const void* D, const void* X, int64_t B, i
     a.X = static_cast<const __nv_bfloat16*>(X);
     a.T = T; a.d = d; a.n = n; a.S = S;
     const dim3 grid((unsigned)((d + 255) / 256), (unsigned)B);
-    if (X) vec_param_kernel<true><<<grid, 256, 0, st>>>(a);
-    else vec_param_kernel<false><<<grid, 256, 0, st>>>(a);
+    if (X) vec_param_kernel<true><<<grid, VP_THREADS, 0, st>>>(a);
+    else vec_param_kernel<false><<<grid, VP_THREADS, 0, st>>>(a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;
