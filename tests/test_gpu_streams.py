@@ -1,0 +1,45 @@
+"""The library enqueues on the caller's stream and keeps contexts independent:
+calls on a non-default stream, two contexts side by side, and results that are
+only read after the stream has been synchronised."""
+import numpy as np
+import pytest
+import torch
+
+import oracle.adloco_oracle as O
+from paper_2508_18182_b200 import binding as A
+from paper_2508_18182_b200 import workloads as W
+from parity import TOL_BF16, TOL_F32, assert_test_result
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def test_non_default_stream_and_two_contexts():
+    c1, c2 = A.Context(0), A.Context(0)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    G1 = W.per_sample_grads(16, 1 << 18, seed=1, device=DEV)
+    G2 = W.per_sample_grads(32, 1 << 17, sigma=1.0, mean_scale="raw", seed=2, device=DEV)
+    X, D = W.linear_layer(4, 256, 128, 256, seed=3, device=DEV)
+    n = torch.zeros(4, device=DEV)
+    S = torch.zeros(256, 128, device=DEV)
+    torch.cuda.synchronize()
+    p1, p2 = A.make_params(0.5, b_cur=16, b_max=32), A.make_params(0.5, b_cur=32, b_max=32)
+    with torch.cuda.stream(s1):
+        c1.norm_test(G1, p1, stream=s1, sync=False)
+        c1.linear_sqnorm(X, D, n, grad_sum=S, method="direct", stream=s1)
+    with torch.cuda.stream(s2):
+        c2.norm_test(G2, p2, stream=s2, sync=False)
+    r1, r2 = c1._read_result(s1), c2._read_result(s2)
+    assert_test_result(r1, O.norm_test(W.to_numpy(G1), eta=0.5, b_cur=16, b_max=32), p1, TOL_F32, what="stream 1")
+    assert_test_result(r2, O.norm_test(W.to_numpy(G2), eta=0.5, b_cur=32, b_max=32), p2, TOL_F32, what="stream 2")
+    n_ref, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
+    assert np.allclose(n.cpu().numpy(), n_ref, rtol=TOL_BF16)
+    assert np.allclose(S.cpu().numpy(), S_ref, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(S_ref).max() * 0.05)
+    c1.close()
+    c2.close()
+
+
+def test_bad_device_index_is_an_error_not_a_crash():
+    with pytest.raises(A.AdlocoError) as e:
+        A.Context(4096)
+    assert e.value.status == A.ERR_CUDA
