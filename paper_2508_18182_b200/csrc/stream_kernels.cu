@@ -369,8 +369,16 @@ static int launch_nt(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
     const size_t smem = (size_t)NT_WARPS * Bpad * sizeof(float);
     auto kern = norm_test_kernel<RB, VEC>;
     if (smem > 48 * 1024) ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int per_sm = 0;
-    ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NT_THREADS, smem));
+    // resident blocks per SM for this instantiation and shared-memory size (asked once)
+    static size_t cached_smem = ~(size_t)0;
+    static int cached_per_sm = 0;
+    if (cached_smem != smem) {
+        int q = 0;
+        ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&q, kern, NT_THREADS, smem));
+        cached_per_sm = q;
+        cached_smem = smem;
+    }
+    const int per_sm = cached_per_sm;
     if (per_sm < 1) return ADLOCO_ERR_WORKSPACE;
     int64_t max_grid = (int64_t)ctx->sm_count * per_sm;
     if (max_grid > ctx->max_grid) max_grid = ctx->max_grid;
@@ -582,8 +590,16 @@ static int launch_ip_t(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
     const size_t smem = (size_t)NT_WARPS * Bpad * sizeof(float);
     auto kern = centred_dot_kernel<RB, VEC>;
     if (smem > 48 * 1024) ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int per_sm = 0;
-    ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NT_THREADS, smem));
+    // resident blocks per SM for this instantiation and shared-memory size (asked once)
+    static size_t cached_smem = ~(size_t)0;
+    static int cached_per_sm = 0;
+    if (cached_smem != smem) {
+        int q = 0;
+        ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&q, kern, NT_THREADS, smem));
+        cached_per_sm = q;
+        cached_smem = smem;
+    }
+    const int per_sm = cached_per_sm;
     if (per_sm < 1) return ADLOCO_ERR_WORKSPACE;
     int64_t max_grid = (int64_t)ctx->sm_count * per_sm;
     if (max_grid > ctx->max_grid) max_grid = ctx->max_grid;
@@ -938,8 +954,17 @@ __global__ void __launch_bounds__(256, 6) outer_step_kernel(const __grid_constan
 // once (so no partial last wave), fewer when the problem is smaller than that.
 template <typename Kern>
 static unsigned elementwise_grid(const adloco_ctx* ctx, Kern kern, int64_t nvec, int threads) {
+    // resident blocks per SM, asked once per kernel
+    static const void* seen[16];
+    static int seen_per_sm[16];
+    static int n_seen = 0;
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    for (int k = 0; k < n_seen; ++k)
+        if (seen[k] == reinterpret_cast<const void*>(kern)) per_sm = seen_per_sm[k];
+    if (per_sm < 1) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+        if (n_seen < 16) { seen[n_seen] = reinterpret_cast<const void*>(kern); seen_per_sm[n_seen] = per_sm; ++n_seen; }
+    }
     int64_t want = (nvec + threads - 1) / threads;
     const int64_t cap = (int64_t)ctx->sm_count * per_sm;
     if (want > cap) want = cap;
