@@ -878,10 +878,12 @@ __device__ __forceinline__ void load_inst4(const void* base, int64_t i, float (&
     }
 }
 
-template <bool BF16, bool WB>
-__global__ void __launch_bounds__(256, 6) outer_step_kernel(const __grid_constant__ OuterArgs a) {
+// KB = instance loads issued back to back: 8 (with registers for them, 4 blocks per SM)
+// when there are at least 8 instances, else 4 (6 blocks per SM) -- measured: K=8 runs 3 %
+// faster with the former, K=4 5 % faster with the latter.
+template <bool BF16, bool WB, int KB>
+__global__ void __launch_bounds__(256, KB == 8 ? 4 : 6) outer_step_kernel(const __grid_constant__ OuterArgs a) {
     constexpr int VEC = 4;
-    constexpr int KB = 4;   // instance loads issued back to back
     const int64_t nvec = a.P / VEC;
     const int64_t step = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
@@ -981,13 +983,16 @@ int launch_outer_step(adloco_ctx* ctx, const OuterLaunch& l, cudaStream_t st) {
     a.th_in = l.th_in; a.th_out = l.th_out; a.v_in = l.v_in; a.v_out = l.v_out;
     a.P = l.P; a.lr = l.lr; a.mu = l.mu; a.invK = 1.0 / (double)l.K; a.K = l.K; a.nesterov = l.nesterov;
     const int64_t nvec = l.P / 4;
-    if (l.bf16) {
-        if (l.has_wb) outer_step_kernel<true, true><<<elementwise_grid(ctx, outer_step_kernel<true, true>, nvec, 256), 256, 0, st>>>(a);
-        else outer_step_kernel<true, false><<<elementwise_grid(ctx, outer_step_kernel<true, false>, nvec, 256), 256, 0, st>>>(a);
+#define ADLOCO_OUTER_LAUNCH(BF, WBK, KBV) \
+    outer_step_kernel<BF, WBK, KBV><<<elementwise_grid(ctx, outer_step_kernel<BF, WBK, KBV>, nvec, 256), 256, 0, st>>>(a)
+    if (l.K >= 8) {
+        if (l.bf16) { if (l.has_wb) ADLOCO_OUTER_LAUNCH(true, true, 8); else ADLOCO_OUTER_LAUNCH(true, false, 8); }
+        else { if (l.has_wb) ADLOCO_OUTER_LAUNCH(false, true, 8); else ADLOCO_OUTER_LAUNCH(false, false, 8); }
     } else {
-        if (l.has_wb) outer_step_kernel<false, true><<<elementwise_grid(ctx, outer_step_kernel<false, true>, nvec, 256), 256, 0, st>>>(a);
-        else outer_step_kernel<false, false><<<elementwise_grid(ctx, outer_step_kernel<false, false>, nvec, 256), 256, 0, st>>>(a);
+        if (l.bf16) { if (l.has_wb) ADLOCO_OUTER_LAUNCH(true, true, 4); else ADLOCO_OUTER_LAUNCH(true, false, 4); }
+        else { if (l.has_wb) ADLOCO_OUTER_LAUNCH(false, true, 4); else ADLOCO_OUTER_LAUNCH(false, false, 4); }
     }
+#undef ADLOCO_OUTER_LAUNCH
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;
