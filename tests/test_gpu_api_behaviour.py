@@ -43,3 +43,33 @@ def test_bad_device_index_is_an_error_not_a_crash():
     with pytest.raises(A.AdlocoError) as e:
         A.Context(4096)
     assert e.value.status == A.ERR_CUDA
+
+
+def test_empty_inputs_are_argument_errors_and_launch_nothing():
+    """Zero-sized problems (no samples, no parameters, no tokens, no instances) are
+    rejected on the host; nothing is enqueued."""
+    import ctypes as C
+    c = A.Context(0)
+    lib, h = c.lib, c.h
+    buf = torch.zeros(1024, device=DEV)
+    bfb = torch.zeros(1024, device=DEV, dtype=torch.bfloat16)
+    p = A.make_params(0.5)
+    before = c.launch_count
+    vp = C.c_void_p
+    d, b = vp(buf.data_ptr()), vp(bfb.data_ptr())
+    res = vp(c._res_dev.data_ptr())
+    assert lib.adloco_norm_test(h, d, A.F32, 0, 16, 16, C.byref(p), None, None, None, res, None, None) == A.ERR_INVALID_ARG
+    assert lib.adloco_norm_test(h, d, A.F32, 4, 0, 0, C.byref(p), None, None, None, res, None, None) == A.ERR_INVALID_ARG
+    assert lib.adloco_norm_test(h, d, A.F32, 4, 16, 8, C.byref(p), None, None, None, res, None, None) == A.ERR_INVALID_ARG  # pitch < P
+    assert lib.adloco_norm_test(h, None, A.F32, 4, 16, 16, C.byref(p), None, None, None, res, None, None) == A.ERR_INVALID_ARG
+    assert lib.adloco_gram_sqnorm(h, b, b, 0, 8, 8, 8, d, 0, None, 0, None) == A.ERR_INVALID_ARG
+    assert lib.adloco_gram_sqnorm(h, b, b, 2, 0, 8, 8, d, 0, None, 0, None) == A.ERR_INVALID_ARG
+    assert lib.adloco_linear_sqnorm(h, b, b, 2, 8, 0, 8, d, 0, None, 0, 0, None) == A.ERR_INVALID_ARG
+    assert lib.adloco_vector_param_sqnorm(h, b, None, 2, 0, 8, d, 0, None, 0, None) == A.ERR_INVALID_ARG
+    arr = (vp * 1)(buf.data_ptr())
+    assert lib.adloco_outer_step(h, arr, A.F32, 0, 16, d, d, d, d, 0.7, 0.9, 1, None, None) == A.ERR_INVALID_ARG
+    assert lib.adloco_outer_step(h, arr, A.F32, 1, 0, d, d, d, d, 0.7, 0.9, 1, None, None) == A.ERR_INVALID_ARG
+    w = (C.c_int64 * 1)(0)
+    assert lib.adloco_merge(h, arr, w, A.F32, 1, 16, d, None, None) == A.ERR_INVALID_ARG      # weight 0
+    assert c.launch_count == before
+    c.close()
