@@ -129,10 +129,11 @@ int adloco_device_status(adloco_ctx* ctx, int32_t* status_host, int clear, void*
 /* Section "Norm test" (Eq. 1, sigma^2_B, b_{k+1}) followed by the switch-mode
  * plan (Section "Mode switching").
  *   grads              dev, [B, P] row-major, row i = g_i, row pitch `row_stride`
- *                      elements (>= P), dtype F32 only.  128-bit loads are used when the
- *                      base is 16-byte aligned and the pitch is a multiple of 4 (and
- *                      grad_sum, if given, is 16-byte aligned); otherwise a slower
- *                      32-bit path runs.  1 <= B <= 4096.
+ *                      elements (>= P), dtype F32 or BF16 (widened exactly, fp32 arithmetic).
+ *                      Vector loads are used when the base is 16-byte (F32) / 8-byte (BF16)
+ *                      aligned and the pitch is a multiple of 4 (and grad_sum, if given, is
+ *                      16-byte aligned); otherwise a slower element-wise path runs.
+ *                      1 <= B <= 4096.
  *   per_sample_sqnorm  dev [B] float, receives n_i = ||g_i||^2; may be NULL
  *   grad_sum           dev [P] float, receives S = sum_i g_i; may be NULL
  *   sums_dev           dev, receives the sufficient statistics; may be NULL

@@ -138,9 +138,9 @@ int adloco_device_status(adloco_ctx* ctx, int32_t* status_host, int clear, void*
 // ---------------------------------------------------------------------------------
 static int check_grads(const void* grads, adloco_dtype dtype, int64_t B, int64_t P, int64_t row_stride) {
     if (!grads || B < 1 || P < 1 || row_stride < P) return ADLOCO_ERR_INVALID_ARG;
-    if (dtype != ADLOCO_F32) return ADLOCO_ERR_UNSUPPORTED;
+    if (dtype != ADLOCO_F32 && dtype != ADLOCO_BF16) return ADLOCO_ERR_UNSUPPORTED;
     if (B > kMaxBatchRows) return ADLOCO_ERR_UNSUPPORTED;
-    if ((reinterpret_cast<uintptr_t>(grads) & 3u) != 0) return ADLOCO_ERR_ALIGNMENT;
+    if ((reinterpret_cast<uintptr_t>(grads) & (dtype == ADLOCO_BF16 ? 1u : 3u)) != 0) return ADLOCO_ERR_ALIGNMENT;
     return ADLOCO_OK;
 }
 
@@ -157,6 +157,7 @@ int adloco_norm_test(adloco_ctx* ctx, const void* grads, adloco_dtype dtype, int
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     NtLaunch l;
     l.G = static_cast<const float*>(grads);
+    l.bf16 = (dtype == ADLOCO_BF16);
     l.B = B; l.P = P; l.stride = row_stride;
     l.n_out = per_sample_sqnorm; l.S = grad_sum;
     l.sums = sums_dev ? sums_dev : ctx->scratch_sums;
@@ -254,6 +255,7 @@ int adloco_inner_product_test(adloco_ctx* ctx, const void* grads, adloco_dtype d
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     IpLaunch l;
     l.G = static_cast<const float*>(grads);
+    l.bf16 = (dtype == ADLOCO_BF16);
     l.S = grad_sum; l.B = B; l.P = P; l.stride = row_stride; l.sums = sums_dev; l.params = *params;
     l.dots_out = inner_products; l.result = result_dev;
     rc = launch_inner_product(ctx, l, st);
@@ -401,6 +403,7 @@ int adloco_accumulate(adloco_ctx* ctx, adloco_accum* a, const void* grads, adloc
     if (a->n_bufs != 1 || a->sizes_host[0] != P) return ADLOCO_ERR_INVALID_ARG;
     NtLaunch l;
     l.G = static_cast<const float*>(grads);
+    l.bf16 = (dtype == ADLOCO_BF16);
     l.B = b_micro; l.P = P; l.stride = row_stride;
     l.n_out = per_sample_sqnorm; l.S = a->bufs_host[0];
     l.sums = a->state; l.result = nullptr; l.mode = NT_MICRO;

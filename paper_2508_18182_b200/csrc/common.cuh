@@ -92,7 +92,8 @@ inline int check_params(const adloco_test_params* p) {
 enum NtMode { NT_ONESHOT = 0, NT_PANEL = 1, NT_MICRO = 2 };
 
 struct NtLaunch {
-    const float* G = nullptr;
+    const float* G = nullptr;     // rows of float, or of bfloat16 when bf16 != 0
+    int bf16 = 0;
     int64_t B = 0, P = 0, stride = 0;
     float* n_out = nullptr;       // [B], may be null
     int n_accum = 0;              // n_out[i] += instead of =
@@ -109,6 +110,7 @@ int launch_decide(adloco_ctx* ctx, const adloco_test_sums* sums, const adloco_te
 
 struct IpLaunch {
     const float* G = nullptr;
+    int bf16 = 0;
     const float* S = nullptr;
     int64_t B = 0, P = 0, stride = 0;
     const adloco_test_sums* sums = nullptr;

@@ -7,6 +7,8 @@
 // arithmetic per byte is far below the machine balance, so grids are sized to
 // a multiple of the SM count and the only tuning that matters is bytes in
 // flight per SM.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace adloco {
@@ -22,6 +24,10 @@ __device__ __forceinline__ float4 ld_stream4(const float* p) {
     return __ldcs(reinterpret_cast<const float4*>(p));
 }
 
+// the two bfloat16 halves of a 32-bit word, widened exactly
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
 // up to four consecutive floats starting at p; lanes >= nvalid read as zero.
 // VEC = false is the path for rows that do not start on a 16-byte boundary.
 template <bool VEC = true>
@@ -32,6 +38,22 @@ __device__ __forceinline__ float4 load4(const float* p, int nvalid) {
     if (nvalid > 0) r.x = __ldcs(p);
     if (nvalid > 1) r.y = __ldcs(p + 1);
     if (nvalid > 2) r.z = __ldcs(p + 2);
+    return r;
+}
+
+// the same for a row of bfloat16: 64-bit load when VEC (rows start on 8-byte boundaries)
+template <bool VEC = true>
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p, int nvalid) {
+    if (VEC && nvalid >= 4) {
+        const uint2 w = __ldcs(reinterpret_cast<const uint2*>(p));
+        return make_float4(bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y));
+    }
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    const unsigned short* q = reinterpret_cast<const unsigned short*>(p);
+    if (nvalid > 0) r.x = __uint_as_float((uint32_t)__ldcs(q) << 16);
+    if (nvalid > 1) r.y = __uint_as_float((uint32_t)__ldcs(q + 1) << 16);
+    if (nvalid > 2) r.z = __uint_as_float((uint32_t)__ldcs(q + 2) << 16);
+    if (nvalid > 3) r.w = __uint_as_float((uint32_t)__ldcs(q + 3) << 16);
     return r;
 }
 
@@ -47,10 +69,6 @@ __device__ __forceinline__ void store4(float* p, float4 v, int nvalid) {
         if (nvalid > 2) p[2] = v.z;
     }
 }
-
-// the two bfloat16 halves of a 32-bit word, widened exactly
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
@@ -188,8 +206,9 @@ struct NtArgs {
 // squares of (G_ij - G_0j) -- shifting by the first row removes the mean before
 // squaring, so the centred sum of squares comes out without cancellation -- and
 // per row the running sum of squares (RB registers, rows tiled by RB).
-template <int RB, bool VEC>
+template <int RB, bool VEC, bool BF16 = false>
 __global__ void __launch_bounds__(NT_THREADS, 2) norm_test_kernel(const __grid_constant__ NtArgs a) {
+    using elem_t = typename std::conditional<BF16, __nv_bfloat16, float>::type;
     extern __shared__ float smem_rows[];  // [NT_WARPS][Bpad]
     __shared__ double smem_red[32];
     __shared__ int smem_is_last;
@@ -221,7 +240,7 @@ __global__ void __launch_bounds__(NT_THREADS, 2) norm_test_kernel(const __grid_c
         const int64_t col = g << 2;
         int nvalid = 0;
         if (g < ngroups) nvalid = (a.P - col) >= 4 ? 4 : (int)(a.P - col);
-        const float* rowp = a.G + (nvalid > 0 ? col : 0);
+        const elem_t* rowp = reinterpret_cast<const elem_t*>(a.G) + (nvalid > 0 ? col : 0);
 
         float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
         float4 sd = c, sdd = c;
@@ -361,13 +380,13 @@ static int grow_workspace(adloco_ctx* ctx, size_t need_elems) {
     return ADLOCO_OK;
 }
 
-template <int RB, bool VEC>
+template <int RB, bool VEC, bool BF16>
 static int launch_nt(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
     const int64_t ngroups = (l.P + 3) / 4;
     const int64_t tiles = (ngroups + NT_THREADS - 1) / NT_THREADS;
     const int Bpad = (int)(((l.B + RB - 1) / RB) * RB);
     const size_t smem = (size_t)NT_WARPS * Bpad * sizeof(float);
-    auto kern = norm_test_kernel<RB, VEC>;
+    auto kern = norm_test_kernel<RB, VEC, BF16>;
     if (smem > 48 * 1024) ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // resident blocks per SM for this instantiation and shared-memory size (asked once)
     static size_t cached_smem = ~(size_t)0;
@@ -400,16 +419,19 @@ static int launch_nt(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
 }
 
 int launch_norm_test(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
-    // 128-bit accesses need every row (and S) to start on a 16-byte boundary
-    const bool vec = aligned16(l.G) && (l.B == 1 || (l.stride % 4) == 0) && (l.S == nullptr || aligned16(l.S));
-    if (vec) {
-        if (l.B <= 16) return launch_nt<16, true>(ctx, l, st);
-        if (l.B <= 32) return launch_nt<32, true>(ctx, l, st);
-        return launch_nt<64, true>(ctx, l, st);
-    }
-    if (l.B <= 16) return launch_nt<16, false>(ctx, l, st);
-    if (l.B <= 32) return launch_nt<32, false>(ctx, l, st);
-    return launch_nt<64, false>(ctx, l, st);
+    // vector loads need every row to start on a 16-byte (fp32) or 8-byte (bf16) boundary, S on 16
+    const uintptr_t row_align = l.bf16 ? 7u : 15u;
+    const bool vec = (reinterpret_cast<uintptr_t>(l.G) & row_align) == 0 && (l.B == 1 || (l.stride % 4) == 0) &&
+                     (l.S == nullptr || aligned16(l.S));
+#define ADLOCO_NT_DISPATCH(V, H)                                         \
+    do {                                                                 \
+        if (l.B <= 16) return launch_nt<16, V, H>(ctx, l, st);           \
+        if (l.B <= 32) return launch_nt<32, V, H>(ctx, l, st);           \
+        return launch_nt<64, V, H>(ctx, l, st);                          \
+    } while (0)
+    if (l.bf16) { if (vec) ADLOCO_NT_DISPATCH(true, true); else ADLOCO_NT_DISPATCH(false, true); }
+    if (vec) ADLOCO_NT_DISPATCH(true, false); else ADLOCO_NT_DISPATCH(false, false);
+#undef ADLOCO_NT_DISPATCH
 }
 
 int launch_decide(adloco_ctx* ctx, const adloco_test_sums* sums, const adloco_test_params& p,
@@ -489,8 +511,9 @@ __device__ void ip_decide_device(double sum_d2, double sum_d, const adloco_test_
 // their entries of S once and walks down the rows accumulating, per row,
 // sum_j (G_ij - S_j / b) S_j = b (<g_i, gbar> - ||gbar||^2): centring before the
 // product keeps the small deviation d_i free of cancellation.
-template <int RB, bool VEC>
+template <int RB, bool VEC, bool BF16 = false>
 __global__ void __launch_bounds__(NT_THREADS, 2) centred_dot_kernel(const __grid_constant__ IpArgs a) {
+    using elem_t = typename std::conditional<BF16, __nv_bfloat16, float>::type;
     extern __shared__ float smem_rows[];  // [NT_WARPS][Bpad]
     __shared__ double smem_red[32];
     __shared__ int smem_is_last;
@@ -514,7 +537,7 @@ __global__ void __launch_bounds__(NT_THREADS, 2) centred_dot_kernel(const __grid
         const int64_t col = g << 2;
         int nvalid = 0;
         if (g < ngroups) nvalid = (a.P - col) >= 4 ? 4 : (int)(a.P - col);
-        const float* rowp = a.G + (nvalid > 0 ? col : 0);
+        const elem_t* rowp = reinterpret_cast<const elem_t*>(a.G) + (nvalid > 0 ? col : 0);
         const float4 s4 = load4<VEC>(a.S + (nvalid > 0 ? col : 0), nvalid);
         const float4 m4 = make_float4(s4.x * invB, s4.y * invB, s4.z * invB, s4.w * invB);
         for (int64_t i0 = 0; i0 < B; i0 += RB) {
@@ -582,13 +605,13 @@ __global__ void __launch_bounds__(NT_THREADS, 2) centred_dot_kernel(const __grid
     }
 }
 
-template <int RB, bool VEC>
+template <int RB, bool VEC, bool BF16>
 static int launch_ip_t(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
     const int64_t ngroups = (l.P + 3) / 4;
     const int64_t tiles = (ngroups + NT_THREADS - 1) / NT_THREADS;
     const int Bpad = (int)(((l.B + RB - 1) / RB) * RB);
     const size_t smem = (size_t)NT_WARPS * Bpad * sizeof(float);
-    auto kern = centred_dot_kernel<RB, VEC>;
+    auto kern = centred_dot_kernel<RB, VEC, BF16>;
     if (smem > 48 * 1024) ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // resident blocks per SM for this instantiation and shared-memory size (asked once)
     static size_t cached_smem = ~(size_t)0;
@@ -618,15 +641,18 @@ static int launch_ip_t(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
 }
 
 int launch_inner_product(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
-    const bool vec = aligned16(l.G) && aligned16(l.S) && (l.B == 1 || (l.stride % 4) == 0);
-    if (vec) {
-        if (l.B <= 16) return launch_ip_t<16, true>(ctx, l, st);
-        if (l.B <= 32) return launch_ip_t<32, true>(ctx, l, st);
-        return launch_ip_t<64, true>(ctx, l, st);
-    }
-    if (l.B <= 16) return launch_ip_t<16, false>(ctx, l, st);
-    if (l.B <= 32) return launch_ip_t<32, false>(ctx, l, st);
-    return launch_ip_t<64, false>(ctx, l, st);
+    const uintptr_t row_align = l.bf16 ? 7u : 15u;
+    const bool vec = (reinterpret_cast<uintptr_t>(l.G) & row_align) == 0 && aligned16(l.S) &&
+                     (l.B == 1 || (l.stride % 4) == 0);
+#define ADLOCO_IP_DISPATCH(V, H)                                         \
+    do {                                                                 \
+        if (l.B <= 16) return launch_ip_t<16, V, H>(ctx, l, st);         \
+        if (l.B <= 32) return launch_ip_t<32, V, H>(ctx, l, st);         \
+        return launch_ip_t<64, V, H>(ctx, l, st);                        \
+    } while (0)
+    if (l.bf16) { if (vec) ADLOCO_IP_DISPATCH(true, true); else ADLOCO_IP_DISPATCH(false, true); }
+    if (vec) ADLOCO_IP_DISPATCH(true, false); else ADLOCO_IP_DISPATCH(false, false);
+#undef ADLOCO_IP_DISPATCH
 }
 
 // ---------------------------------------------------------------------------------

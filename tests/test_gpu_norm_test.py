@@ -131,9 +131,10 @@ def test_argument_errors_never_launch(ctx):
         with pytest.raises(A.AdlocoError) as e:
             ctx.norm_test(G, bad)
         assert e.value.status == A.ERR_INVALID_ARG
-    with pytest.raises(A.AdlocoError) as e:
-        ctx.norm_test(torch.zeros(4, 64, device=DEV, dtype=torch.bfloat16), A.make_params(0.5))
-    assert e.value.status == A.ERR_UNSUPPORTED
+    import ctypes as C
+    rc = ctx.lib.adloco_norm_test(ctx.h, C.c_void_p(G.data_ptr()), 7, 4, 64, 64, C.byref(A.make_params(0.5)), None, None,
+                                  None, C.c_void_p(ctx._res_dev.data_ptr()), None, None)       # no such dtype
+    assert rc == A.ERR_UNSUPPORTED
     with pytest.raises(A.AdlocoError) as e:
         ctx.norm_test(torch.zeros(4097, 8, device=DEV), A.make_params(0.5))
     assert e.value.status == A.ERR_UNSUPPORTED
@@ -147,6 +148,39 @@ def test_unaligned_rows_take_the_scalar_path(ctx):
     _check(ctx, G, A.make_params(0.5, b_cur=3, b_max=32), "unaligned")
     G2 = W.per_sample_grads(70, 4103, seed=7, device=DEV, row_stride=4105)
     _check(ctx, G2, A.make_params(0.5, b_cur=70, b_max=32), "odd pitch")
+
+
+@pytest.mark.parametrize("B,P,stride", [(16, 1 << 18, None), (3, 4099, None), (64, 70001, 70004), (65, 9001, None),
+                                        (33, 12345, 12348)])
+def test_bf16_gradients(ctx, B, P, stride):
+    """Per-sample gradients stored as bfloat16 are widened exactly; the oracle reads the same bits."""
+    G32 = W.per_sample_grads(B, P, sigma=0.5, seed=B, device=DEV, row_stride=stride)
+    buf = torch.zeros((B, stride or P), dtype=torch.bfloat16, device=DEV)
+    G = buf[:, :P]
+    G.copy_(G32)
+    p = A.make_params(0.5, b_cur=B, b_max=32)
+    n = torch.zeros(B, device=DEV)
+    S = torch.zeros(P, device=DEV)
+    r = ctx.norm_test(G, p, per_sample_sqnorm=n, grad_sum=S)
+    ora = O.norm_test(W.to_numpy(G.contiguous()), eta=0.5, b_cur=B, b_max=32, want_sum=True)
+    assert_test_result(r, ora, p, TOL_F32, what=f"bf16 B={B} P={P}")
+    assert np.allclose(n.cpu().numpy(), ora.per_sample_sqnorm, rtol=TOL_F32)
+    assert np.allclose(S.cpu().numpy(), ora.grad_sum, rtol=1e-5, atol=1e-5 * B)
+    # switch-mode accumulation of the same rows in two micro-batches
+    if B >= 2 and stride is None:
+        h = B // 2
+        Sacc = torch.empty(P, device=DEV)
+        acc = A.Accumulator(ctx, [Sacc])
+        acc.reset()
+        acc.accumulate(G[:h].contiguous())
+        acc.accumulate(G[h:].contiguous())
+        ra = acc.finalize(p)
+        assert_test_result(ra, ora, p, TOL_F32, what="bf16 accumulated")
+        acc.close()
+    # inner-product tests on the bf16 rows
+    ri = ctx.inner_product_test(G, S, theta=0.01, nu=0.3, b_cur=B)
+    oi = O.inner_product_tests(W.to_numpy(G.contiguous()), theta=0.01, nu=0.3, b_cur=B)
+    assert rel_close(ri.stat_ip, oi.stat_ip, 4 * TOL_F32) and rel_close(ri.stat_orth, oi.stat_orth, 4 * TOL_F32)
 
 
 def test_largest_supported_batch(ctx):
