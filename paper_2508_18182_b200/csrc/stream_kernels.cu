@@ -207,8 +207,9 @@ struct NtArgs {
 // squaring, so the centred sum of squares comes out without cancellation -- and
 // per row the running sum of squares (RB registers, rows tiled by RB).
 template <int RB, bool VEC, bool BF16 = false>
-__global__ void __launch_bounds__(NT_THREADS, 2) norm_test_kernel(const __grid_constant__ NtArgs a) {
+__global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(const __grid_constant__ NtArgs a) {
     using elem_t = typename std::conditional<BF16, __nv_bfloat16, float>::type;
+    constexpr int CH = RB < NT_CHUNK ? RB : NT_CHUNK;   // rows loaded back to back
     extern __shared__ float smem_rows[];  // [NT_WARPS][Bpad]
     __shared__ double smem_red[32];
     __shared__ int smem_is_last;
@@ -246,16 +247,16 @@ __global__ void __launch_bounds__(NT_THREADS, 2) norm_test_kernel(const __grid_c
         float4 sd = c, sdd = c;
         for (int64_t i0 = 0; i0 < B; i0 += RB) {
 #pragma unroll
-            for (int r0 = 0; r0 < RB; r0 += NT_CHUNK) {
-                float4 x[NT_CHUNK];
+            for (int r0 = 0; r0 < RB; r0 += CH) {
+                float4 x[CH];
 #pragma unroll
-                for (int u = 0; u < NT_CHUNK; ++u) {
+                for (int u = 0; u < CH; ++u) {
                     const bool ok = (i0 + r0 + u) < B;
                     x[u] = load4<VEC>(rowp + (int64_t)(r0 + u) * a.stride, ok ? nvalid : 0);
                 }
                 if (i0 == 0 && r0 == 0) c = x[0];
 #pragma unroll
-                for (int u = 0; u < NT_CHUNK; ++u) {
+                for (int u = 0; u < CH; ++u) {
                     if ((i0 + r0 + u) < B) {
                         const float4 v = x[u];
                         float q = v.x * v.x;
@@ -425,6 +426,8 @@ int launch_norm_test(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
                      (l.S == nullptr || aligned16(l.S));
 #define ADLOCO_NT_DISPATCH(V, H)                                         \
     do {                                                                 \
+        if (l.B <= 4) return launch_nt<4, V, H>(ctx, l, st);             \
+        if (l.B <= 8) return launch_nt<8, V, H>(ctx, l, st);             \
         if (l.B <= 16) return launch_nt<16, V, H>(ctx, l, st);           \
         if (l.B <= 32) return launch_nt<32, V, H>(ctx, l, st);           \
         return launch_nt<64, V, H>(ctx, l, st);                          \
@@ -512,8 +515,9 @@ __device__ void ip_decide_device(double sum_d2, double sum_d, const adloco_test_
 // sum_j (G_ij - S_j / b) S_j = b (<g_i, gbar> - ||gbar||^2): centring before the
 // product keeps the small deviation d_i free of cancellation.
 template <int RB, bool VEC, bool BF16 = false>
-__global__ void __launch_bounds__(NT_THREADS, 2) centred_dot_kernel(const __grid_constant__ IpArgs a) {
+__global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) centred_dot_kernel(const __grid_constant__ IpArgs a) {
     using elem_t = typename std::conditional<BF16, __nv_bfloat16, float>::type;
+    constexpr int CH = RB < NT_CHUNK ? RB : NT_CHUNK;   // rows loaded back to back
     extern __shared__ float smem_rows[];  // [NT_WARPS][Bpad]
     __shared__ double smem_red[32];
     __shared__ int smem_is_last;
@@ -542,15 +546,15 @@ __global__ void __launch_bounds__(NT_THREADS, 2) centred_dot_kernel(const __grid
         const float4 m4 = make_float4(s4.x * invB, s4.y * invB, s4.z * invB, s4.w * invB);
         for (int64_t i0 = 0; i0 < B; i0 += RB) {
 #pragma unroll
-            for (int r0 = 0; r0 < RB; r0 += NT_CHUNK) {
-                float4 x[NT_CHUNK];
+            for (int r0 = 0; r0 < RB; r0 += CH) {
+                float4 x[CH];
 #pragma unroll
-                for (int u = 0; u < NT_CHUNK; ++u) {
+                for (int u = 0; u < CH; ++u) {
                     const bool ok = (i0 + r0 + u) < B;
                     x[u] = load4<VEC>(rowp + (int64_t)(r0 + u) * a.stride, ok ? nvalid : 0);
                 }
 #pragma unroll
-                for (int u = 0; u < NT_CHUNK; ++u) {
+                for (int u = 0; u < CH; ++u) {
                     if ((i0 + r0 + u) < B) {
                         // columns beyond P carry s4 = 0 and add nothing
                         float q = (x[u].x - m4.x) * s4.x;
@@ -646,6 +650,8 @@ int launch_inner_product(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
                      (l.B == 1 || (l.stride % 4) == 0);
 #define ADLOCO_IP_DISPATCH(V, H)                                         \
     do {                                                                 \
+        if (l.B <= 4) return launch_ip_t<4, V, H>(ctx, l, st);           \
+        if (l.B <= 8) return launch_ip_t<8, V, H>(ctx, l, st);           \
         if (l.B <= 16) return launch_ip_t<16, V, H>(ctx, l, st);         \
         if (l.B <= 32) return launch_ip_t<32, V, H>(ctx, l, st);         \
         return launch_ip_t<64, V, H>(ctx, l, st);                        \
