@@ -305,11 +305,19 @@ int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
     if (!ctx || !X || !D || !per_sample_sqnorm) return ADLOCO_ERR_INVALID_ARG;
     if (B < 1 || T < 1 || d_in < 1 || d_out < 1) return ADLOCO_ERR_INVALID_ARG;
     if (method == ADLOCO_LINEAR_AUTO) {
-        // tensor work of the two routes, at the granularity the kernels execute
+        // tensor work of the two routes at the granularity the kernels execute, divided by
+        // the share of the SMs their work items can occupy (few tokens give the Gram kernel
+        // fewer items than there are SMs; the direct kernel then wins despite more flops)
+        const double sms = (double)ctx->sm_count;
         const double nt = (double)((T + 127) / 128);
-        const double gram = 2.0 * (double)B * (nt * (nt + 1) / 2) * 128.0 * 128.0 * (double)(d_in + d_out) +
-                            (grad_sum ? 2.0 * (double)B * (double)T * (double)d_in * (double)d_out : 0.0);
-        const double direct = 2.0 * (double)B * (double)T * (double)d_in * (double)d_out;
+        const double gram_items = (double)B * ((nt * (nt + 1) / 2 + 1) / 2);           // about one item per two blocks
+        const double dir_items = (double)((d_out + 127) / 128) * (double)((d_in + 255) / 256) * (double)B;
+        const double gemm = 2.0 * (double)B * (double)T * (double)d_in * (double)d_out;
+        const double gram_util = gram_items < sms ? gram_items / sms : 1.0;
+        const double dir_util = dir_items < sms ? dir_items / sms : 1.0;
+        const double gram = 2.0 * (double)B * (nt * (nt + 1) / 2) * 128.0 * 128.0 * (double)(d_in + d_out) / gram_util +
+                            (grad_sum ? gemm / dir_util : 0.0);
+        const double direct = gemm / dir_util;
         method = direct <= gram ? ADLOCO_LINEAR_DIRECT : ADLOCO_LINEAR_GRAM;
     }
     if (method == ADLOCO_LINEAR_GRAM)
