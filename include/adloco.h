@@ -33,7 +33,7 @@
 extern "C" {
 #endif
 
-typedef struct adloco_ctx adloco_ctx;     /* device id, workspace, cached tensor maps */
+typedef struct adloco_ctx adloco_ctx;     /* device id and workspace */
 typedef struct adloco_accum adloco_accum; /* switch-mode accumulator state */
 
 typedef enum {

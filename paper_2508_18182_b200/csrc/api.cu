@@ -96,7 +96,6 @@ int adloco_create(adloco_ctx** out, int device) {
 int adloco_destroy(adloco_ctx* ctx) {
     if (!ctx) return ADLOCO_ERR_INVALID_ARG;
     DeviceGuard g(ctx->device);
-    free_tmap_cache(ctx);
     cudaFree(ctx->n_partials);
     cudaFree(ctx->blk_scalars);
     cudaFree(ctx->ticket);

@@ -48,9 +48,6 @@ struct adloco_ctx {
     float* n_scratch = nullptr;                // [kMaxBatchRows] per-sample norms when the caller wants none
 
     adloco::HostStaging staging;
-
-    // cached TMA descriptors of the tensor-core path (opaque here)
-    void* tmap_cache = nullptr;
 };
 
 struct adloco_accum {
@@ -162,6 +159,5 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
 int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                          int64_t d_out, float* n, int accumulate_norms, float* S, int accumulate_sum,
                          cudaStream_t st);
-void free_tmap_cache(adloco_ctx* ctx);
 
 }  // namespace adloco

@@ -765,10 +765,10 @@ int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     a.total_items = (int)((fulls + halves) * B);
     a.n = n; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {false};   // the attribute is per device
+    if (!attr_set[ctx->device & 63]) {
         ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(gram_sqnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GR_SMEM));
-        attr_set = true;
+        attr_set[ctx->device & 63] = true;
     }
     const int grid = a.total_items < ctx->sm_count ? a.total_items : ctx->sm_count;
     gram_sqnorm_kernel<<<grid, GR_THREADS, GR_SMEM, st>>>(tmX, tmD, a);
@@ -793,10 +793,10 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
     a.splits = sp.splits; a.chunk = sp.chunk; a.items = sp.items;
     a.S = S; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {false};   // the attribute is per device
+    if (!attr_set[ctx->device & 63]) {
         ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(mean_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM));
-        attr_set = true;
+        attr_set[ctx->device & 63] = true;
     }
     const int grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
     mean_grad_kernel<<<grid, MG_THREADS, MG_SMEM, st>>>(tmX, tmD, a);
@@ -823,10 +823,10 @@ int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
     a.n = n; a.S = S; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
     if (S && !accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {false};   // the attribute is per device
+    if (!attr_set[ctx->device & 63]) {
         ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(direct_sqnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_SMEM));
-        attr_set = true;
+        attr_set[ctx->device & 63] = true;
     }
     const int grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
     direct_sqnorm_kernel<<<grid, DR_THREADS, DR_SMEM, st>>>(tmX, tmD, a);
@@ -835,6 +835,5 @@ int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
     return ADLOCO_OK;
 }
 
-void free_tmap_cache(adloco_ctx*) {}
 
 }  // namespace adloco
