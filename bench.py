@@ -546,6 +546,22 @@ def run_table(args):
          oracle_note="one block x one micro-batch timed, x48 extrapolated")
     ms4d = gpu_ms(lambda: whole_model("auto"), reps=5, warm=1)
     emit(4, "whole model, linear_sqnorm auto (direct route)", ms4d, flops=f_mg, oracle_s=o4, oracle_note="as above")
+    # the same 192 calls captured once into a CUDA graph and replayed (nothing in them synchronises)
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            whole_model("auto")
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            whole_model("auto")
+        ms4g = gpu_ms(graph.replay, reps=5, warm=1)
+        emit(4, "whole model, direct route, replayed as one CUDA graph", ms4g, flops=f_mg, oracle_s=o4, oracle_note="as above")
+        del graph
+    except Exception as exc:   # capture is an extra, not part of the path
+        print(json.dumps({"config": 4, "kernel": "CUDA graph replay", "skipped": str(exc)[:200]}), flush=True)
     acc.close()
     del data, sums
     torch.cuda.empty_cache()

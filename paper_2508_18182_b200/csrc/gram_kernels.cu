@@ -286,7 +286,9 @@ constexpr int MG_BOX_BYTES = 64 * MG_BK * 2;        // one TMA box: 64 features 
 constexpr int MG_A_BYTES = (MG_BM / 64) * MG_BOX_BYTES;
 constexpr int MG_B_BYTES = (MG_BN / 64) * MG_BOX_BYTES;
 constexpr int MG_STAGE_BYTES = MG_A_BYTES + MG_B_BYTES;   // 64 KB
-constexpr int MG_SMEM = MG_STAGES * MG_STAGE_BYTES + 1024 + 256;
+constexpr int MG_BOX_OUT = 32 * 32 * 4;             // per-epilogue-warp staging box: 32 rows x 32 fp32 columns
+constexpr int MG_STAGING = 8 * MG_BOX_OUT;
+constexpr int MG_SMEM = MG_STAGES * MG_STAGE_BYTES + MG_STAGING + 1024 + 256;
 constexpr int MG_THREADS = 320;                     // warp 0 TMA, warp 1 MMA, warps 2-9 epilogue
 
 struct MeanGradArgs {
@@ -300,10 +302,11 @@ struct MeanGradArgs {
 
 __global__ void __launch_bounds__(MG_THREADS, 1)
 mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
-                 const MeanGradArgs a) {
+                 const __grid_constant__ CUtensorMap tmS, const MeanGradArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bar_base = smem_base + MG_STAGES * MG_STAGE_BYTES;
+    const uint32_t staging_base = smem_base + MG_STAGES * MG_STAGE_BYTES;   // 1024-aligned
+    const uint32_t bar_base = staging_base + MG_STAGING;
     auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
     auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (MG_STAGES + s); };
     const uint32_t tfull_bar = bar_base + 8u * (2 * MG_STAGES);
@@ -322,6 +325,7 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         fence_barrier_init();
         prefetch_tmap(&tmX);
         prefetch_tmap(&tmD);
+        prefetch_tmap(&tmS);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&tmem_base_slot), 512);   // rows 0-127 in columns 0-255, rows 128-255 in 256-511
@@ -437,27 +441,30 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar, seg & 1u, abortp, a.wait_ns))) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((q * 32u) << 16) + half * 256u;
-            const int m = tm * MG_BM + (int)half * 128 + (int)q * 32 + lane;
-            float* srow = a.S + (int64_t)m * a.d_in;
+            const int m0 = tm * MG_BM + (int)half * 128 + (int)q * 32;   // first of this warp's 32 rows
+            // The tile goes to S in 32x32 boxes: the warp writes a box to shared memory (lane =
+            // row, 128-byte swizzle) and one TMA reduction adds it into S as full 128-byte lines;
+            // rows and columns outside S are dropped by the hardware.
+            const uint32_t box = staging_base + (uint32_t)(warp - 2) * MG_BOX_OUT;
+            const uint32_t row_addr = box + (uint32_t)lane * 128u;
 #pragma unroll 1
             for (int cc = 0; cc < MG_BN / 32; ++cc) {
                 uint32_t r[32];
                 tmem_ld32(taddr + cc * 32, r);
                 tmem_ld_wait();
                 const int n0 = tn * MG_BN + cc * 32;
-                if (m < a.d_out && n0 < a.d_in) {
+                if (m0 < a.d_out && n0 < a.d_in) {            // uniform across the warp
+                    if (lane == 0) bulk_wait_read_all();      // the previous box has been read
+                    __syncwarp();
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        const int n = n0 + e;
-                        if (n + 3 < a.d_in) {
-                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(srow + n),
-                                         "f"(__uint_as_float(r[e])), "f"(__uint_as_float(r[e + 1])),
-                                         "f"(__uint_as_float(r[e + 2])), "f"(__uint_as_float(r[e + 3]))
-                                         : "memory");
-                        } else {
-                            for (int z = 0; z < 4; ++z)
-                                if (n + z < a.d_in) atomicAdd(srow + n + z, __uint_as_float(r[e + z]));
-                        }
+                    for (int j = 0; j < 8; ++j)
+                        st_shared_v4(row_addr + (uint32_t)((j ^ (lane & 7)) << 4), r[4 * j], r[4 * j + 1], r[4 * j + 2],
+                                     r[4 * j + 3]);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_reduce_add_2d(&tmS, box, n0, m0);
+                        bulk_commit_group();
                     }
                 }
             }
@@ -468,6 +475,8 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             ++seg;
         }
         }
+        if (lane == 0) bulk_wait_all();   // this warp's reductions into S are complete
+        __syncwarp();
     }
 
     tc_fence_before();
@@ -496,7 +505,9 @@ constexpr int DR_BOX_BYTES = 64 * DR_BK * 2;        // 8 KB
 constexpr int DR_A_BYTES = (DR_BM / 64) * DR_BOX_BYTES;
 constexpr int DR_B_BYTES = (DR_BN / 64) * DR_BOX_BYTES;
 constexpr int DR_STAGE_BYTES = DR_A_BYTES + DR_B_BYTES;   // 48 KB
-constexpr int DR_SMEM = DR_STAGES * DR_STAGE_BYTES + 1024 + 256;
+constexpr int DR_BOX_OUT = 32 * 16 * 4;             // per-epilogue-warp staging box: 32 rows x 16 fp32 columns
+constexpr int DR_STAGING = 12 * DR_BOX_OUT;
+constexpr int DR_SMEM = DR_STAGES * DR_STAGE_BYTES + DR_STAGING + 1024 + 256;
 // Epilogue: three warps per TMEM lane quarter; the 16 column chunks (of 16) of a tile
 // row are split 6 / 5 / 5 among them, so a thread keeps at most 96 columns of the S
 // tile in registers (16 warps' worth of register file at 128 registers per thread).
@@ -517,10 +528,11 @@ struct DirectArgs {
 
 __global__ void __launch_bounds__(DR_THREADS, 1)
 direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
-                     const DirectArgs a) {
+                     const __grid_constant__ CUtensorMap tmS, const DirectArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bar_base = smem_base + DR_STAGES * DR_STAGE_BYTES;
+    const uint32_t staging_base = smem_base + DR_STAGES * DR_STAGE_BYTES;
+    const uint32_t bar_base = staging_base + DR_STAGING;
     auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
     auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (DR_STAGES + s); };
     auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * DR_STAGES + b); };
@@ -538,6 +550,7 @@ direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         fence_barrier_init();
         prefetch_tmap(&tmX);
         prefetch_tmap(&tmD);
+        if (a.S != nullptr) prefetch_tmap(&tmS);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&tmem_base_slot), 512);   // two 128x256 fp32 accumulators
@@ -670,29 +683,39 @@ direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const float w = warp_sum_f(sq);
                 if (lane == 0) atomicAdd(a.n + i, w);
             }
-            // end of the segment: add this thread's part of the tile's row into S
+            // end of the segment: add this warp's 32 rows x its column slice into S, 16 columns
+            // at a time: the warp lays a 32 x 16 box out in shared memory (lane = row) and one TMA
+            // reduction adds it into S; rows and columns outside S are dropped by the hardware
             const int tm = tile / a.ntn, tn = tile % a.ntn;
-            const int m = tm * DR_BM + (int)q * 32 + lane;
-            const int n0 = tn * DR_BN + c_begin * 16;
-            float* srow = a.S + (int64_t)m * a.d_in;
-            const bool row_ok = ok && a.S != nullptr && m < a.d_out;
+            const int m0 = tm * DR_BM + (int)q * 32;
+            const int n_base = tn * DR_BN + c_begin * 16;
+            const uint32_t box = staging_base + (uint32_t)(warp - 2) * DR_BOX_OUT;
+            const uint32_t row_addr = box + (uint32_t)lane * 64u;
+            const bool flush = ok && a.S != nullptr && m0 < a.d_out;     // uniform across the warp
 #pragma unroll
-            for (int e = 0; e < DR_COLS; e += 4) {
-                const int n = n0 + e;
-                if (row_ok && e < n_chunks * 16) {
-                    if (n + 3 < a.d_in) {
-                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(srow + n),
-                                     "f"(sacc[e]), "f"(sacc[e + 1]), "f"(sacc[e + 2]), "f"(sacc[e + 3]) : "memory");
-                    } else {
+            for (int cc = 0; cc < DR_CHUNKS_MAX; ++cc) {
+                if (flush && cc < n_chunks && n_base + cc * 16 < a.d_in) {
+                    if (lane == 0) bulk_wait_read_all();                 // the previous box has been read
+                    __syncwarp();
 #pragma unroll
-                        for (int z = 0; z < 4; ++z)
-                            if (n + z < a.d_in) atomicAdd(srow + n + z, sacc[e + z]);
+                    for (int j = 0; j < 4; ++j)
+                        st_shared_v4(row_addr + (uint32_t)(j << 4), __float_as_uint(sacc[cc * 16 + 4 * j]),
+                                     __float_as_uint(sacc[cc * 16 + 4 * j + 1]), __float_as_uint(sacc[cc * 16 + 4 * j + 2]),
+                                     __float_as_uint(sacc[cc * 16 + 4 * j + 3]));
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_reduce_add_2d(&tmS, box, n_base + cc * 16, m0);
+                        bulk_commit_group();
                     }
                 }
-                sacc[e] = 0.f; sacc[e + 1] = 0.f; sacc[e + 2] = 0.f; sacc[e + 3] = 0.f;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) sacc[cc * 16 + e] = 0.f;
             }
         }
         }
+        if (lane == 0) bulk_wait_all();   // this warp's reductions into S are complete
+        __syncwarp();
     }
 
     tc_fence_before();
@@ -745,6 +768,25 @@ static int make_map(adloco_ctx* ctx, CUtensorMap* m, const void* base, int64_t B
     return ADLOCO_OK;
 }
 
+// fp32 matrix [rows, cols] (cols contiguous) as a 2-D map with a 32-row box of box_cols
+// columns: 32 columns with the 128-byte swizzle, 16 columns unswizzled
+static int make_map_f32(adloco_ctx* ctx, CUtensorMap* m, float* base, int64_t rows, int64_t cols, uint32_t box_cols) {
+    EncodeTiledFn fn = encode_fn(ctx);
+    if (!fn) return ADLOCO_ERR_CUDA;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+    const cuuint32_t box[2] = {box_cols, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    box_cols == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(ctx->cuda_err, sizeof(ctx->cuda_err), "cuTensorMapEncodeTiled (fp32) failed with CUresult %d", (int)r);
+        return ADLOCO_ERR_CUDA;
+    }
+    return ADLOCO_OK;
+}
+
 int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                        int64_t d_out, float* n, int accumulate_norms, cudaStream_t st) {
     CUtensorMap tmX, tmD;
@@ -784,6 +826,9 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
     if (rc != ADLOCO_OK) return rc;
     rc = make_map(ctx, &tmD, D, B, T, d_out, MG_BK);
     if (rc != ADLOCO_OK) return rc;
+    CUtensorMap tmS;
+    rc = make_map_f32(ctx, &tmS, S, d_out, d_in, 32);
+    if (rc != ADLOCO_OK) return rc;
     MeanGradArgs a;
     a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
     a.ntm = (int)((d_out + MG_BM - 1) / MG_BM);
@@ -799,7 +844,7 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
         attr_set[ctx->device & 63] = true;
     }
     const int grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
-    mean_grad_kernel<<<grid, MG_THREADS, MG_SMEM, st>>>(tmX, tmD, a);
+    mean_grad_kernel<<<grid, MG_THREADS, MG_SMEM, st>>>(tmX, tmD, tmS, a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;
@@ -813,6 +858,13 @@ int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
     if (rc != ADLOCO_OK) return rc;
     rc = make_map(ctx, &tmD, D, B, T, d_out, DR_BK);
     if (rc != ADLOCO_OK) return rc;
+    CUtensorMap tmS;
+    if (S) {
+        rc = make_map_f32(ctx, &tmS, S, d_out, d_in, 16);
+        if (rc != ADLOCO_OK) return rc;
+    } else {
+        tmS = tmX;   // never used by the kernel when S is null
+    }
     DirectArgs a;
     a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
     a.ntm = (int)((d_out + DR_BM - 1) / DR_BM);
@@ -829,7 +881,7 @@ int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
         attr_set[ctx->device & 63] = true;
     }
     const int grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
-    direct_sqnorm_kernel<<<grid, DR_THREADS, DR_SMEM, st>>>(tmX, tmD, a);
+    direct_sqnorm_kernel<<<grid, DR_THREADS, DR_SMEM, st>>>(tmX, tmD, tmS, a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;
