@@ -274,6 +274,24 @@ def vector_param_terms(D, X=None):
     return n, S
 
 
+def embedding_terms(ids, D, V: int):
+    """Per-sample gradients of an embedding table E [V, d] looked up at every token:
+    row v of sample i's gradient is the sum of delta_{i,t} over the tokens t with
+    ids[i, t] = v.  ids [B, T] integers in [0, V), D [B, T, d].
+    Returns n_i = ||G_i||_F^2 and S = sum_i G_i ([V, d])."""
+    ids = np.asarray(ids)
+    B = ids.shape[0]
+    d = D.shape[2]
+    n = np.zeros(B, dtype=np.float64)
+    S = np.zeros((V, d), dtype=np.float64)
+    for i in range(B):
+        G_i = np.zeros((V, d), dtype=np.float64)
+        np.add.at(G_i, ids[i], widen(D[i]))
+        n[i] = float(np.sum(G_i * G_i))
+        S += G_i
+    return n, S
+
+
 def linear_layers_norm_test(layers, *, eta: float, ddof: int = 1, b_cur: int = 1,
                             b_max: int = 1, b_cap: int = 0, switch_n: int = 2,
                             two_pass: bool = True) -> NormTestResult:

@@ -222,6 +222,39 @@ def pin_vector_param_terms(O):
     assert np.array_equal(n_lin, n) and np.array_equal(S_lin[:, 0], S)
 
 
+def pin_embedding_terms(O):
+    rng = np.random.default_rng(23)
+    _, D = W.small_integer_layer(3, 7, 8, 8, seed=31)
+    Dn, Di = W.to_numpy(D), D.float().numpy()
+    V = 5
+    ids = rng.integers(0, V, size=(3, 7))
+    n, S = O.embedding_terms(ids, Dn, V)
+    S_ref = [[0] * 8 for _ in range(V)]
+    for i in range(3):
+        G = [[0] * 8 for _ in range(V)]
+        for t in range(7):
+            for j in range(8):
+                G[int(ids[i, t])][j] += int(Di[i][t][j])
+        assert n[i] == float(sum(x * x for row in G for x in row))
+        for v in range(V):
+            for j in range(8):
+                S_ref[v][j] += G[v][j]
+    assert S.tolist() == [[float(x) for x in row] for row in S_ref]
+    # a lookup is a linear layer on one-hot inputs: same per-sample norms, transposed sum
+    onehot = torch.zeros(3, 7, V, dtype=torch.bfloat16)
+    for i in range(3):
+        for t in range(7):
+            onehot[i, t, int(ids[i, t])] = 1.0
+    n_lin, S_lin = O.linear_layer_terms(W.to_numpy(onehot), Dn)
+    assert np.array_equal(n_lin, n) and np.array_equal(S_lin.T, S)
+    # all tokens distinct: n_i = sum_t ||delta_t||^2; all equal: the bias case
+    n_d, _ = O.embedding_terms(np.tile(np.arange(7), (3, 1)), Dn, 7)
+    assert np.array_equal(n_d, (Di.astype(np.float64) ** 2).sum(axis=(1, 2)))
+    n_e, S_e = O.embedding_terms(np.full((3, 7), 2), Dn, 4)
+    n_b, S_b = O.vector_param_terms(Dn)
+    assert np.array_equal(n_e, n_b) and np.array_equal(S_e[2], S_b) and not S_e[[0, 1, 3]].any()
+
+
 def pin_layers_test_two_routes(O):
     layers = [tuple(W.to_numpy(t) for t in W.linear_layer(4, 6, 8, 16, seed=1)),
               tuple(W.to_numpy(t) for t in W.linear_layer(4, 6, 16, 8, seed=2))]
@@ -396,6 +429,7 @@ MUTANTS = [
     ("merge takes the largest", "order = sorted(range(k), key=lambda i: (b_req[i], i))",
      "order = sorted(range(k), key=lambda i: (-b_req[i], i))"),
     ("merge unweighted", "x += float(b) * widen(p)", "x += widen(p)"),
+    ("embedding rows overwritten instead of summed", "np.add.at(G_i, ids[i], widen(D[i]))", "G_i[ids[i]] = widen(D[i])"),
     ("vector parameter summed over features", "g = (d * widen(X[i])).sum(axis=0) if X is not None else d.sum(axis=0)",
      "g = (d * widen(X[i])).sum(axis=1) if X is not None else d.sum(axis=1)"),
     ("gain gradient without the input", "g = (d * widen(X[i])).sum(axis=0) if X is not None else d.sum(axis=0)",
