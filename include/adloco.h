@@ -268,6 +268,20 @@ int adloco_vector_param_sqnorm(adloco_ctx* ctx, const void* D, const void* X, in
                                float* per_sample_sqnorm, int accumulate_norms, float* grad_sum, int accumulate_sum,
                                void* stream);
 
+/* Per-sample gradient norms of an embedding table E [V, d] looked up at every token
+ * (Eq. 1 applied to E): row v of sample i's gradient is the sum of delta_{i,t} over the
+ * tokens with token_ids[i, t] = v, so n_i = sum_{t,s} [id_t == id_s] (delta_t . delta_s)
+ * -- the Gram identity with a token-equality mask in place of X X^T, on the tensor cores.
+ * With position indices as ids it covers a learned positional embedding.
+ *   token_ids          dev int32 [B, T], values in [0, V) (others match nothing and are skipped)
+ *   D                  dev bf16 [B, T, d]: gradient of the loss w.r.t. the looked-up rows; d % 8 == 0
+ *   per_sample_sqnorm  dev [B] float; overwritten, or += when accumulate_norms != 0
+ *   grad_sum           dev [V, d] float, may be NULL: S = sum_i G_i (scatter-add); overwritten
+ *                      (V d floats are cleared first), or += when accumulate_sum != 0 */
+int adloco_embedding_sqnorm(adloco_ctx* ctx, const int32_t* token_ids, const void* D, int64_t B, int64_t T, int64_t d,
+                            int64_t V, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
+                            int accumulate_sum, void* stream);
+
 /* ---- switch-mode accumulation -------------------------------------------- */
 
 /* Accumulator of the test sums over the micro-batches of one large batch:

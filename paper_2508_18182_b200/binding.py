@@ -23,7 +23,7 @@ FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN = 1, 2, 4, 8
 EXPORTS = (
     "adloco_create", "adloco_destroy", "adloco_status_string", "adloco_last_cuda_error", "adloco_launch_count",
     "adloco_set_wait_limit", "adloco_device_status",
-    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_inner_product_test", "adloco_gram_sqnorm", "adloco_linear_sqnorm", "adloco_vector_param_sqnorm",
+    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_inner_product_test", "adloco_gram_sqnorm", "adloco_linear_sqnorm", "adloco_vector_param_sqnorm", "adloco_embedding_sqnorm",
     "adloco_accum_create", "adloco_accum_reset", "adloco_accum_destroy", "adloco_accumulate",
     "adloco_accum_finalize", "adloco_outer_step", "adloco_outer_step_host", "adloco_check_merge", "adloco_merge",
 )
@@ -97,6 +97,7 @@ def load_library() -> C.CDLL:
         "adloco_gram_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
         "adloco_linear_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, C.c_int, vp]),
         "adloco_vector_param_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
+        "adloco_embedding_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
         "adloco_accum_create": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), i32]),
         "adloco_accum_reset": (C.c_int, [vp, vp, vp]),
         "adloco_accum_destroy": (C.c_int, [vp]),
@@ -277,6 +278,18 @@ class Context:
                                                  int(accumulate_norms), _ptr(grad_sum), int(accumulate_sum),
                                                  _stream(stream))
         self.check(rc, "adloco_vector_param_sqnorm")
+
+    def embedding_sqnorm(self, token_ids, D, V, per_sample_sqnorm, *, accumulate_norms=False, grad_sum=None,
+                         accumulate_sum=False, stream=None):
+        """adloco_embedding_sqnorm: token_ids int32 [B, T], D bf16 [B, T, d], table of V rows."""
+        B, T, d = D.shape
+        if token_ids.dtype != torch.int32 or tuple(token_ids.shape) != (B, T) or not token_ids.is_contiguous():
+            raise AdlocoError(ERR_INVALID_ARG, "token_ids must be contiguous int32 [B, T]")
+        if D.dtype != torch.bfloat16 or not D.is_contiguous():
+            raise AdlocoError(ERR_INVALID_ARG, "D must be contiguous bfloat16")
+        rc = self.lib.adloco_embedding_sqnorm(self.h, _ptr(token_ids), _ptr(D), B, T, d, int(V), _ptr(per_sample_sqnorm),
+                                              int(accumulate_norms), _ptr(grad_sum), int(accumulate_sum), _stream(stream))
+        self.check(rc, "adloco_embedding_sqnorm")
 
     # ------------------------------------------------------------------ outer step
     def outer_step(self, instances, theta_in, mom_in, *, lr, momentum, nesterov=True, theta_out=None,

@@ -296,6 +296,19 @@ int adloco_vector_param_sqnorm(adloco_ctx* ctx, const void* D, const void* X, in
                             static_cast<cudaStream_t>(stream));
 }
 
+int adloco_embedding_sqnorm(adloco_ctx* ctx, const int32_t* token_ids, const void* D, int64_t B, int64_t T, int64_t d,
+                            int64_t V, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
+                            int accumulate_sum, void* stream) {
+    if (!ctx || !token_ids || !D || !per_sample_sqnorm) return ADLOCO_ERR_INVALID_ARG;
+    if (B < 1 || T < 1 || d < 1 || V < 1) return ADLOCO_ERR_INVALID_ARG;
+    if ((d % 8) != 0 || B > (1 << 30) || T > (1 << 30) || d > (1 << 30) || V > 0x7fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    if (!aligned16(D) || (reinterpret_cast<uintptr_t>(token_ids) & 3u) != 0) return ADLOCO_ERR_ALIGNMENT;
+    if (grad_sum && !aligned16(grad_sum)) return ADLOCO_ERR_ALIGNMENT;
+    DeviceGuard g(ctx->device);
+    return launch_embedding(ctx, token_ids, D, B, T, d, V, per_sample_sqnorm, accumulate_norms, grad_sum, accumulate_sum,
+                            static_cast<cudaStream_t>(stream));
+}
+
 int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                          int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
                          int accumulate_sum, int method, void* stream) {

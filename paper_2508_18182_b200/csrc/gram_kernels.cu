@@ -245,6 +245,190 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
 }
 
+// =====================================================================================
+// embedding kernel: Gram identity with the activations' Gram matrix replaced by a mask
+// =====================================================================================
+// Sample i's gradient of an embedding table has row v = sum of delta_t over the tokens
+// with id_t = v, so ||G_i||^2 = sum_{t,s} [id_t == id_s] (delta_t . delta_s): the Gram
+// kernel without the X X^T product -- the epilogue keeps the entries of D D^T whose two
+// tokens carry the same id.  Same work items (sample, row tile, one or two column
+// blocks on or above the diagonal); the accumulator is double-buffered.
+struct EmbedArgs {
+    GramArgs g;          // B, T, d_out = embedding width, item bookkeeping, n, status, wait bound
+    const int* ids;      // [B, T]
+};
+
+__global__ void __launch_bounds__(GR_THREADS, 1)
+embed_gram_kernel(const __grid_constant__ CUtensorMap tmD, const EmbedArgs ea) {
+    const GramArgs& a = ea.g;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_base = smem_base + GR_STAGES * GR_STAGE_BYTES;
+    auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (GR_STAGES + s); };
+    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * GR_STAGES + b); };
+    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * GR_STAGES + 2 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * GR_STAGES + 4);
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (uint32_t s = 0; s < GR_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+        mbar_init(drain_bar, 1);
+        fence_barrier_init();
+        prefetch_tmap(&tmD);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);   // two 128x256 accumulators of D D^T
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+    const int chunks = (a.d_out + GR_BK - 1) / GR_BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            PipeState ps;
+            uint32_t issued = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < a.total_items; item += gridDim.x) {
+                int i, ti, c0, ncb;
+                gram_decode(item, a, i, ti, c0, ncb);
+                const bool diag = (c0 == ti);
+                for (int c = 0; c < chunks; ++c) {
+                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
+                    const uint32_t sA = smem_base + ps.stage * GR_STAGE_BYTES;
+                    mbar_arrive_expect_tx(full_bar(ps.stage), ((diag ? 0 : 1) + ncb) * GR_BLOCK_BYTES);
+                    if (!diag) tma_load_3d(sA, &tmD, full_bar(ps.stage), c * GR_BK, ti * GR_TILE, i);
+                    tma_load_3d(sA + GR_BLOCK_BYTES, &tmD, full_bar(ps.stage), c * GR_BK, c0 * GR_TILE, i);
+                    if (ncb == 2)
+                        tma_load_3d(sA + 2 * GR_BLOCK_BYTES, &tmD, full_bar(ps.stage), c * GR_BK, (c0 + 1) * GR_TILE, i);
+                    ++issued;
+                    ps.advance(GR_STAGES);
+                }
+            }
+            if (!ok) {
+                PipeState q = ps;
+                const uint32_t back = issued < GR_STAGES ? issued : GR_STAGES;
+                for (uint32_t r = 0; r < back; ++r) {
+                    if (q.stage == 0) { q.stage = GR_STAGES - 1; q.phase ^= 1u; } else { --q.stage; }
+                    int never = 0;
+                    mbar_wait(full_bar(q.stage), q.phase, &never, kDrainLimitNs);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            PipeState ps;
+            bool ok = true;
+            int n_item = 0;
+            for (int item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++n_item) {
+                int i, ti, c0, ncb;
+                gram_decode(item, a, i, ti, c0, ncb);
+                const uint32_t idesc = idesc_bf16_f32(GR_TILE, GR_TILE * ncb, 0, 0);
+                const uint32_t buf = n_item & 1, use = n_item >> 1;
+                if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t acc = tmem_base + buf * 256u;
+                for (int c = 0; c < chunks; ++c) {
+                    if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, a.wait_ns)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sB = smem_base + ps.stage * GR_STAGE_BYTES + GR_BLOCK_BYTES;
+                    const uint32_t sA = (c0 == ti) ? sB : sB - GR_BLOCK_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < GR_BK / 16; ++kk) {
+                        const uint64_t da = smem_desc_sw128(sA + kk * 32, 16, 1024);
+                        const uint64_t db = smem_desc_sw128(sB + kk * 32, 16, 1024);
+                        mma_bf16(acc, da, db, idesc, (c == 0 && kk == 0) ? 0u : 1u);
+                    }
+                    mma_commit(empty_bar(ps.stage));
+                    ps.advance(GR_STAGES);
+                }
+                if (ok) mma_commit(tfull_bar(buf));
+            }
+            if (!ok) {
+                mma_commit(drain_bar);
+                int never = 0;
+                mbar_wait(drain_bar, 0, &never, kDrainLimitNs);
+            }
+        }
+    } else {
+        const uint32_t q = warp & 3;
+        const uint32_t half = (warp - 2) >> 2;
+        int n_item = 0;
+        for (int item = blockIdx.x; item < a.total_items; item += gridDim.x, ++n_item) {
+            int i, ti, c0, ncb;
+            gram_decode(item, a, i, ti, c0, ncb);
+            // ids of this thread's row and of the columns it will visit; tokens beyond T never match
+            const int* ids_i = ea.ids + (int64_t)i * a.T;
+            const int t_row = ti * GR_TILE + (int)q * 32 + lane;
+            const int id_row = t_row < a.T ? __ldg(ids_i + t_row) : -1;
+            const uint32_t buf = n_item & 1, use = n_item >> 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abortp, a.wait_ns))) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + buf * 256u;
+            const int cols_per_half = 64 * ncb;
+            const int col_begin = (int)half * cols_per_half;
+            float sum = 0.f;
+#pragma unroll 1
+            for (int col = col_begin; col < col_begin + cols_per_half; col += 32) {
+                uint32_t d[32];
+                tmem_ld32(taddr + col, d);
+                const int t_col = c0 * GR_TILE + col + lane;                 // lane l holds the id of column col + l
+                const int id_col = t_col < a.T ? __ldg(ids_i + t_col) : -2;
+                tmem_ld_wait();
+                float part = 0.f;
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    part += (__shfl_sync(0xffffffffu, id_col, e) == id_row) ? __uint_as_float(d[e]) : 0.f;
+                sum += (c0 + (col >> 7) == ti) ? part : 2.0f * part;
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            const float w = warp_sum_f(sum);
+            if (lane == 0) atomicAdd(a.n + i, w);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
+}
+
+// S[id_t, :] += delta_t for every token: one warp per token row, 128-bit loads, vector reductions
+__global__ void __launch_bounds__(256) embed_scatter_kernel(const int* ids, const __nv_bfloat16* D, int64_t tokens,
+                                                            int d, int V, float* S) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp_global = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t t = warp_global; t < tokens; t += n_warps) {
+        const int id = __ldg(ids + t);
+        if (id < 0 || id >= V) continue;             // ids outside the table are ignored
+        const __nv_bfloat16* row = D + t * d;
+        float* dst = S + (int64_t)id * d;
+        for (int f = lane * 8; f < d; f += 256) {    // d is a multiple of 8
+            const uint4 w = __ldcs(reinterpret_cast<const uint4*>(row + f));
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + f),
+                         "f"(__uint_as_float(w.x << 16)), "f"(__uint_as_float(w.x & 0xffff0000u)),
+                         "f"(__uint_as_float(w.y << 16)), "f"(__uint_as_float(w.y & 0xffff0000u)) : "memory");
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + f + 4),
+                         "f"(__uint_as_float(w.z << 16)), "f"(__uint_as_float(w.z & 0xffff0000u)),
+                         "f"(__uint_as_float(w.w << 16)), "f"(__uint_as_float(w.w & 0xffff0000u)) : "memory");
+        }
+    }
+}
+
 // Work split shared by the two token-contraction kernels.  The (tile, sample) units of
 // one output tile are cut into `splits` chunks of `chunk` consecutive samples, every
 // chunk starting at a multiple of `chunk`; work item j = (tile j / splits, chunk
@@ -816,6 +1000,49 @@ int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     gram_sqnorm_kernel<<<grid, GR_THREADS, GR_SMEM, st>>>(tmX, tmD, a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
+    return ADLOCO_OK;
+}
+
+int launch_embedding(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, int64_t T, int64_t d, int64_t V,
+                     float* n, int accumulate_norms, float* S, int accumulate_sum, cudaStream_t st) {
+    CUtensorMap tmD;
+    int rc = make_map(ctx, &tmD, D, B, T, d, GR_TILE);
+    if (rc != ADLOCO_OK) return rc;
+    EmbedArgs ea;
+    GramArgs& a = ea.g;
+    a.B = (int)B; a.T = (int)T; a.d_in = 0; a.d_out = (int)d;
+    a.nt = (int)((T + GR_TILE - 1) / GR_TILE);
+    int64_t fulls = 0;
+    for (int ti = 0; ti < a.nt; ++ti) fulls += (a.nt - ti) / 2;
+    const int64_t halves = (a.nt + 1) / 2;
+    if ((fulls + halves) * B > 0x7fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    a.full_per_sample = (int)fulls;
+    a.half_per_sample = (int)halves;
+    a.n_full = (int)(fulls * B);
+    a.total_items = (int)((fulls + halves) * B);
+    a.n = n; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
+    ea.ids = ids;
+    if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
+    static bool attr_set[64] = {false};   // the attribute is per device
+    if (!attr_set[ctx->device & 63]) {
+        ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(embed_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GR_SMEM));
+        attr_set[ctx->device & 63] = true;
+    }
+    const int grid = a.total_items < ctx->sm_count ? a.total_items : ctx->sm_count;
+    embed_gram_kernel<<<grid, GR_THREADS, GR_SMEM, st>>>(tmD, ea);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    if (S) {
+        if (!accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)V * (size_t)d * sizeof(float), st));
+        const int64_t tokens = B * T;
+        int64_t blocks = (tokens + 7) / 8;
+        const int64_t cap = (int64_t)ctx->sm_count * 8;
+        if (blocks > cap) blocks = cap;
+        embed_scatter_kernel<<<(unsigned)blocks, 256, 0, st>>>(ids, static_cast<const __nv_bfloat16*>(D), tokens, (int)d,
+                                                               (int)V, S);
+        ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+        ctx->launches++;
+    }
     return ADLOCO_OK;
 }
 
