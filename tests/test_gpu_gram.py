@@ -160,3 +160,50 @@ def test_a_wait_that_runs_out_raises_the_status_and_the_context_stays_usable(met
     assert np.allclose(n.cpu().numpy(), n_ref, rtol=TOL_BF16)
     assert np.allclose(S.cpu().numpy(), S_ref, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(S_ref).max() * 0.05)
     c.close()
+
+
+def test_every_parameter_kind_in_one_accumulated_test(ctx):
+    """A small transformer-shaped parameter set -- token and positional embeddings, a
+    LayerNorm gain and bias, two linear layers with biases -- tested as one model over two
+    micro-batches.  The oracle materialises every per-sample gradient, concatenates them
+    and applies the definition of the norm test."""
+    B, n_micro, T, d, V = 4, 2, 96, 64, 30
+    sizes = {"tok": (V, d), "pos": (T, d), "ln_g": (d,), "ln_b": (d,), "w1": (128, d), "b1": (128,), "w2": (d, 128), "b2": (d,)}
+    S = {k: torch.empty(*shape, device=DEV) for k, shape in sizes.items()}
+    acc = A.Accumulator(ctx, list(S.values()))
+    acc.reset()
+    pos = torch.arange(T, device=DEV, dtype=torch.int32).repeat(B, 1).contiguous()
+    flat = []
+    for j in range(n_micro):
+        g = torch.Generator(device=DEV)
+        g.manual_seed(500 + j)
+        ids = torch.randint(0, V, (B, T), generator=g, device=DEV, dtype=torch.int32)
+        Xh, De = W.linear_layer(B, T, d, d, seed=10 + j, delta_std=0.3, device=DEV)      # normalised input, grad at the embedding / LN output
+        X1, D1 = W.linear_layer(B, T, d, 128, seed=20 + j, delta_std=0.1, device=DEV)
+        X2, D2 = W.linear_layer(B, T, 128, d, seed=30 + j, delta_std=0.1, device=DEV)
+        n = torch.zeros(B, device=DEV)
+        ctx.embedding_sqnorm(ids, De, V, n, grad_sum=S["tok"], accumulate_sum=True)
+        ctx.embedding_sqnorm(pos, De, T, n, accumulate_norms=True, grad_sum=S["pos"], accumulate_sum=True)
+        ctx.vector_param_sqnorm(De, n, X=Xh, accumulate_norms=True, grad_sum=S["ln_g"], accumulate_sum=True)
+        ctx.vector_param_sqnorm(De, n, accumulate_norms=True, grad_sum=S["ln_b"], accumulate_sum=True)
+        ctx.linear_sqnorm(X1, D1, n, accumulate_norms=True, grad_sum=S["w1"], accumulate_sum=True, method="gram")
+        ctx.vector_param_sqnorm(D1, n, accumulate_norms=True, grad_sum=S["b1"], accumulate_sum=True)
+        ctx.linear_sqnorm(X2, D2, n, accumulate_norms=True, grad_sum=S["w2"], accumulate_sum=True, method="direct")
+        ctx.vector_param_sqnorm(D2, n, accumulate_norms=True, grad_sum=S["b2"], accumulate_sum=True)
+        acc.accumulate(per_sample_sqnorm=n)
+        # the oracle's explicit per-sample gradients, in the same parameter order
+        idn, De_n, Xh_n = ids.cpu().numpy(), O.widen(W.to_numpy(De)), O.widen(W.to_numpy(Xh))
+        for i in range(B):
+            tok = np.zeros((V, d)); np.add.at(tok, idn[i], De_n[i])
+            parts = [tok.ravel(), De_n[i].ravel(), (De_n[i] * Xh_n[i]).sum(0), De_n[i].sum(0),
+                     O.per_sample_weight_grad(W.to_numpy(X1[i]), W.to_numpy(D1[i])).ravel(), O.widen(W.to_numpy(D1[i])).sum(0),
+                     O.per_sample_weight_grad(W.to_numpy(X2[i]), W.to_numpy(D2[i])).ravel(), O.widen(W.to_numpy(D2[i])).sum(0)]
+            flat.append(np.concatenate(parts))
+    p = A.make_params(0.5, b_cur=B * n_micro, b_max=B)
+    r = acc.finalize(p)
+    ora = O.norm_test(np.stack(flat), eta=0.5, b_cur=B * n_micro, b_max=B, want_sum=True)
+    kappa = ora.sum_sqnorm / max(ora.variance * (B * n_micro - 1), 1e-300)
+    assert_test_result(r, ora, p, TOL_BF16, stat_tol=TOL_BF16 * max(1.0, kappa), what="all parameter kinds")
+    got = np.concatenate([S[k].cpu().numpy().ravel() for k in sizes])
+    assert np.allclose(got, ora.grad_sum, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(ora.grad_sum).max() * 0.05)
+    acc.close()
