@@ -517,6 +517,17 @@ def run_table(args):
     Dn8 = Dn[:8]
     emit(3, "vector_param_sqnorm (bias of the layer, Delta [32,1024,3072])", ms_b, nbytes=2 * GR_B * GR_T * GR_DOUT,
          oracle_s=cpu_s(lambda: O.vector_param_terms(Dn8)) * 4, oracle_note="8 samples timed, x4", note="L2 flushed")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4)
+    ids = torch.randint(0, 50257, (GR_B, GR_T), generator=gen, device=dev, dtype=torch.int32)
+    De = X                                               # [32, 1024, 768] bf16 stands in for the output gradient
+    Se = torch.zeros(50257, GR_DIN, device=dev)
+    ms_e = gpu_ms(lambda: ctx.embedding_sqnorm(ids, De, 50257, n))
+    ms_es = gpu_ms(lambda: ctx.embedding_sqnorm(ids, De, 50257, n, grad_sum=Se, accumulate_sum=True))
+    emit(3, "embedding_sqnorm (norms only; ids [32,1024], V=50257, d=768)", ms_e, flops=GR_B * GR_T * (GR_T + 1) * GR_DIN)
+    emit(3, "embedding scatter-add of the gradient sum (difference)", ms_es - ms_e,
+         nbytes=GR_B * GR_T * GR_DIN * (2 + 4), note="2 bytes read + 4 bytes added per element")
+    del Se
     # config 4: 12 blocks x 4 layers x 4 micro-batches, all inputs resident (38.7 GB)
     shapes = list(W.GPT2_SMALL_BLOCK_LINEARS) * 12
     data = [[W.linear_layer(32, 1024, di, do, seed=1000 * j + l, device=dev) for l, (di, do) in enumerate(shapes)]
@@ -546,6 +557,30 @@ def run_table(args):
          oracle_note="one block x one micro-batch timed, x48 extrapolated")
     ms4d = gpu_ms(lambda: whole_model("auto"), reps=5, warm=1)
     emit(4, "whole model, linear_sqnorm auto (direct route)", ms4d, flops=f_mg, oracle_s=o4, oracle_note="as above")
+    # the layers of a micro-batch are independent (they only add into n and into their own S): issued
+    # alternately on two streams, the tail of one layer's kernel overlaps the head of the next
+    s_a, s_b = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def whole_model_two_streams():
+        main = torch.cuda.current_stream()
+        acc.reset()
+        for j in range(4):
+            n_mb.zero_()                                   # every layer adds into n with atomics
+            s_a.wait_stream(main)
+            s_b.wait_stream(main)
+            for l, (Xl, Dl) in enumerate(data[j]):
+                ctx.linear_sqnorm(Xl, Dl, n_mb, accumulate_norms=True, grad_sum=sums[l], accumulate_sum=True,
+                                  method="auto", stream=(s_a if (l & 1) == 0 else s_b))
+            main.wait_stream(s_a)
+            main.wait_stream(s_b)
+            acc.accumulate(per_sample_sqnorm=n_mb)
+        acc.finalize(p4, sync=False)
+    try:
+        ms4s = gpu_ms(whole_model_two_streams, reps=5, warm=1)
+        emit(4, "whole model, direct route, layers alternating on two streams", ms4s, flops=f_mg, oracle_s=o4,
+             oracle_note="as above")
+    except Exception as exc:
+        print(json.dumps({"config": 4, "kernel": "two streams", "skipped": str(exc)[:200]}), flush=True)
     # the same 192 calls captured once into a CUDA graph and replayed (nothing in them synchronises)
     try:
         side = torch.cuda.Stream()

@@ -18,8 +18,15 @@
  *     16-byte aligned unless an entry point says otherwise (ADLOCO_ERR_ALIGNMENT
  *     if not).  The library owns only the workspace inside an adloco_ctx.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
- *     legacy default stream) and is asynchronous unless stated.  One ctx must
- *     not be used from two streams at the same time: its workspace is shared.
+ *     legacy default stream) and is asynchronous unless stated.  The streaming
+ *     entry points (norm test, accumulate, finalize, inner-product test, host
+ *     variants) share the ctx workspace: do not run two of them at the same
+ *     time on one ctx.  The tensor-core entry points (adloco_gram_sqnorm,
+ *     adloco_linear_sqnorm, adloco_embedding_sqnorm), adloco_vector_param_sqnorm,
+ *     adloco_outer_step and adloco_merge use none of it and may be issued on
+ *     several streams at once -- the layers of one micro-batch only add into
+ *     n and into their own S, and alternating them on two streams overlaps
+ *     one kernel's tail with the next one's start.
  *   - Sizes are int64_t element counts; all byte offsets are 64-bit inside.
  *   - There is no CPU fallback: without a usable CUDA device the calls fail
  *     with ADLOCO_ERR_CUDA.
