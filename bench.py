@@ -77,9 +77,9 @@ def aggregate_throughput(units_per_rank: float, world: int, max_seconds: float) 
 
 
 # DRAM traffic of norm_test_kernel per gradient element, from the ncu capture of the
-# profiling case (B=64, P=2^21: 536.98 MB read + 4.28 MB written for 2^27 elements);
+# profiling case (B=64, P=2^21: 536.98 MB read + 4.10 MB written for 2^27 elements);
 # traffic grows in proportion to B*P, so a full launch is this times its element count.
-NT_TRAFFIC_BYTES_PER_ELEMENT = (536.978e6 + 4.280e6) / float(64 * (1 << 21))
+NT_TRAFFIC_BYTES_PER_ELEMENT = (536.98e6 + 4.10e6) / float(64 * (1 << 21))
 
 
 def load_peaks():
