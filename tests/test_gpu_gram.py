@@ -56,6 +56,8 @@ def test_small_integer_layer_is_exact(ctx, method):
     (1, 384, 768, 256),      # 3x3 token tiles, 12 + 4 chunks: the ring wraps
     (4, 130, 264, 520),      # d_in > 256 and d_out > 512: several output tiles, ragged
     (33, 64, 32, 48),
+    (2, 2048, 256, 512),     # long sequence: 16 token blocks per side, 72 tile items per sample
+    (1, 1153, 64, 64),       # odd number of blocks (10) with a ragged last one
 ])
 @pytest.mark.parametrize("method", METHODS)
 def test_layer_matches_oracle(ctx, B, T, d_in, d_out, method):
