@@ -50,7 +50,9 @@ constexpr int GR_STAGES = 4;
 constexpr int GR_BLOCK_BYTES = GR_TILE * GR_BK * 2;          // 16 KB: 128 rows of one stage
 constexpr int GR_STAGE_BYTES = 3 * GR_BLOCK_BYTES;           // row tile + up to two column blocks
 constexpr int GR_SMEM = GR_STAGES * GR_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
-constexpr int GR_THREADS = 320;                              // warp 0 TMA, warp 1 MMA, warps 2-9 epilogue
+constexpr int GR_EPI_WARPS = 8;                              // epilogue warps: GR_PARTS per TMEM lane quarter
+constexpr int GR_PARTS = GR_EPI_WARPS / 4;                   // each takes 1/GR_PARTS of the tile's columns
+constexpr int GR_THREADS = 64 + 32 * GR_EPI_WARPS;           // warp 0 TMA, warp 1 MMA, the rest epilogue
 
 struct GramArgs {
     int B, T, d_in, d_out;
@@ -105,7 +107,7 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         abort_flag = 0;
         for (uint32_t s = 0; s < GR_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(tfull_bar, 1);
-        mbar_init(tempty_bar, 8);
+        mbar_init(tempty_bar, GR_EPI_WARPS);
         mbar_init(drain_bar, 1);
         fence_barrier_init();
         prefetch_tmap(&tmX);
@@ -203,7 +205,7 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     } else {
         // ---------------- epilogue: sum over the tile of (X X^T) .* (D D^T) ----------------
         const uint32_t q = warp & 3;            // TMEM lanes 32q .. 32q+31 belong to this warp
-        const uint32_t half = (warp - 2) >> 2;  // which half of the tile's columns
+        const uint32_t half = (warp - 2) >> 2;  // which part of the tile's columns
         int n_item = 0;
         for (int item = blockIdx.x; item < a.total_items; item += gridDim.x, ++n_item) {
             int i, ti, c0, ncb;
@@ -212,7 +214,7 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar, n_item & 1u, abortp, a.wait_ns))) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((q * 32u) << 16);
-            const int cols_per_half = 64 * ncb;
+            const int cols_per_half = (GR_TILE * ncb) / GR_PARTS;
             const int col_begin = (int)half * cols_per_half;
             float sum = 0.f;
 #pragma unroll 1
@@ -276,7 +278,7 @@ embed_gram_kernel(const __grid_constant__ CUtensorMap tmD, const EmbedArgs ea) {
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (uint32_t s = 0; s < GR_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+        for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), GR_EPI_WARPS); }
         mbar_init(drain_bar, 1);
         fence_barrier_init();
         prefetch_tmap(&tmD);
@@ -373,7 +375,7 @@ embed_gram_kernel(const __grid_constant__ CUtensorMap tmD, const EmbedArgs ea) {
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abortp, a.wait_ns))) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((q * 32u) << 16) + buf * 256u;
-            const int cols_per_half = 64 * ncb;
+            const int cols_per_half = (GR_TILE * ncb) / GR_PARTS;
             const int col_begin = (int)half * cols_per_half;
             float sum = 0.f;
 #pragma unroll 1
