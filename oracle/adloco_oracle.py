@@ -30,9 +30,13 @@ choice):
 Pins (tests/test_oracle_pins.py): exact rational brute force on tiny integer
 inputs, closed forms (orthonormal gradients, rank-one layer, zero momentum),
 the LocalSGD average as a special case of the outer step, a hand-worked dyadic
-example, and invariances.  The momentum convention and ddof are conventions
-the paper does not fix: for those two choices parity is unpinned beyond the
-closed forms that follow from the reading itself.
+example, agreement with the library's SGD optimiser, and invariances; every
+function in this file has at least one such pin.  Two readings cannot be
+settled from the paper's text -- the variance normaliser (ddof) and the
+momentum form of OuterOpt: both are parameters here, each value of them is
+pinned (ddof 0 and 1 by the closed forms, Nesterov and heavy-ball momentum by
+the library optimiser and the hand-worked example), and which one the authors
+meant is recorded as a reading in the design notes.
 """
 from __future__ import annotations
 
