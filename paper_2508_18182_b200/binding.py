@@ -345,6 +345,33 @@ def norm_test_noalloc(G, params: TestParams, result_dev, result_host, *, per_sam
     return TestResult.from_buffer_copy(result_host.numpy().tobytes()[:C.sizeof(TestResult)])
 
 
+def shard_bounds(P: int, rank: int, world: int, align: int = 8):
+    """[begin, end) of rank `rank`'s slice when a flat parameter vector of P elements is
+    cut into `world` contiguous slices whose starts are multiples of `align` elements
+    (8 keeps fp32 and bf16 slices 16-byte aligned).  The slices are disjoint and cover
+    [0, P); trailing ranks may get an empty slice when P is small."""
+    if not (0 <= rank < world) or P < 0 or align < 1:
+        raise ValueError("bad shard request")
+    units = -(-P // align)
+    lo = min(P, (units * rank // world) * align)
+    hi = min(P, (units * (rank + 1) // world) * align)
+    return lo, hi
+
+
+def outer_step_shard(ctx, instances, theta, mom, rank: int, world: int, *, lr, momentum, nesterov=True,
+                     writeback=None, stream=None):
+    """The outer step on this rank's slice of the parameter vector.  The update is
+    elementwise, so when every GPU holds its slice of theta, of the momentum and of all K
+    instances, the sharded outer step needs no exchange at all: each rank calls this on its
+    own buffers (here: views into full-length tensors).  Returns the slice bounds."""
+    lo, hi = shard_bounds(theta.numel(), rank, world)
+    if hi > lo:
+        wb = None if writeback is None else [None if t is None else t[lo:hi] for t in writeback]
+        ctx.outer_step([t[lo:hi] for t in instances], theta[lo:hi], mom[lo:hi], lr=lr, momentum=momentum,
+                       nesterov=nesterov, writeback=wb, stream=stream)
+    return lo, hi
+
+
 def TestResult_size() -> int:
     return C.sizeof(TestResult)
 

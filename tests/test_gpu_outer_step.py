@@ -124,3 +124,20 @@ def test_merge_matches_oracle(ctx, dtype):
     # merging into one of the members, exactly aliased
     ctx.merge(inst, weights, inst[1])
     assert torch.equal(inst[1], out)
+
+
+@pytest.mark.parametrize("world", [2, 3, 8])
+def test_sharded_outer_step_equals_the_whole(ctx, world):
+    """Every rank updating its own slice (no exchange: the update is elementwise) gives
+    bit for bit the result of the unsharded call.  The ranks' kernels are independent; they
+    are simply run one after the other here."""
+    theta, inst, mom = W.outer_state(4, 100003, inst_dtype=torch.bfloat16, seed=77, device=DEV, zero_momentum=False)
+    th_ref, v_ref = ctx.outer_step(inst, theta.clone(), mom.clone(), lr=0.7, momentum=0.9)
+    th, v = theta.clone(), mom.clone()
+    covered = 0
+    for r in range(world):
+        lo, hi = A.outer_step_shard(ctx, inst, th, v, r, world, lr=0.7, momentum=0.9)
+        assert lo == covered
+        covered = hi
+    assert covered == theta.numel()
+    assert torch.equal(th, th_ref) and torch.equal(v, v_ref)

@@ -50,3 +50,17 @@ def test_single_process_is_the_identity():
     assert bench.aggregate_throughput(4.0, 1, 2.0) == 2.0
     nt, outer = bench.algorithmic_bytes()
     assert nt == 4 * 64 * (1 << 24) and outer == (2 * 8 + 16) * 124_439_808
+
+
+def test_shard_bounds_partition_the_vector():
+    from paper_2508_18182_b200.binding import shard_bounds
+    for P in (0, 1, 7, 8, 9, 1000, 124_439_808, 1_300_000_000, 12345677):
+        for world in (1, 2, 3, 4, 8, 13):
+            prev = 0
+            for r in range(world):
+                lo, hi = shard_bounds(P, r, world)
+                assert lo == prev and hi >= lo and (lo % 8 == 0 or lo == P)
+                prev = hi
+            assert prev == P
+            sizes = [shard_bounds(P, r, world)[1] - shard_bounds(P, r, world)[0] for r in range(world)]
+            assert max(sizes) - min(sizes) <= 8 + 7        # balanced to within one aligned unit
