@@ -300,7 +300,7 @@ int adloco_accum_create(adloco_ctx* ctx, adloco_accum** out, float* const* sum_b
                         int32_t n_bufs);
 /* Zeroes Q, the count and every S buffer (async on stream). */
 int adloco_accum_reset(adloco_ctx* ctx, adloco_accum* acc, void* stream);
-int adloco_accum_destroy(adloco_accum* acc);
+int adloco_accum_destroy(adloco_accum* acc);   /* before its ctx is destroyed */
 
 /* Adds one micro-batch (Algorithm 3's g <- g + grad L(x; B), applied to the
  * test sums).  Two forms:

@@ -13,6 +13,8 @@
 // memory into TMEM accumulators, the remaining warps drain the accumulators.
 // Every wait is bounded; a wait that runs out raises a status word and all
 // roles leave through the common teardown.
+#include <atomic>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -921,16 +923,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn encode_fn(adloco_ctx* ctx) {
-    static EncodeTiledFn fn = nullptr;
-    if (fn) return fn;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
-    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) {
-        set_cuda_error(ctx, e != cudaSuccess ? e : cudaErrorUnknown, "cuTensorMapEncodeTiled entry point");
-        return nullptr;
-    }
-    fn = reinterpret_cast<EncodeTiledFn>(p);
+    // looked up once; the initialisation of a function-local static is thread-safe
+    static const EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        const cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+        if (e != cudaSuccess || q != cudaDriverEntryPointSuccess) return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    if (!fn) set_cuda_error(ctx, cudaErrorUnknown, "cuTensorMapEncodeTiled entry point");
     return fn;
 }
 
@@ -993,10 +994,10 @@ int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     a.total_items = (int)((fulls + halves) * B);
     a.n = n; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
-    static bool attr_set[64] = {false};   // the attribute is per device
-    if (!attr_set[ctx->device & 63]) {
+    static std::atomic<bool> attr_set[64];   // the attribute is per device
+    if (!attr_set[ctx->device & 63].load()) {
         ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(gram_sqnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GR_SMEM));
-        attr_set[ctx->device & 63] = true;
+        attr_set[ctx->device & 63].store(true);
     }
     const int grid = a.total_items < ctx->sm_count ? a.total_items : ctx->sm_count;
     gram_sqnorm_kernel<<<grid, GR_THREADS, GR_SMEM, st>>>(tmX, tmD, a);
@@ -1025,10 +1026,10 @@ int launch_embedding(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, 
     a.n = n; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     ea.ids = ids;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
-    static bool attr_set[64] = {false};   // the attribute is per device
-    if (!attr_set[ctx->device & 63]) {
+    static std::atomic<bool> attr_set[64];   // the attribute is per device
+    if (!attr_set[ctx->device & 63].load()) {
         ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(embed_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GR_SMEM));
-        attr_set[ctx->device & 63] = true;
+        attr_set[ctx->device & 63].store(true);
     }
     const int grid = a.total_items < ctx->sm_count ? a.total_items : ctx->sm_count;
     embed_gram_kernel<<<grid, GR_THREADS, GR_SMEM, st>>>(tmD, ea);
@@ -1067,10 +1068,10 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
     a.splits = sp.splits; a.chunk = sp.chunk; a.items = sp.items;
     a.S = S; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
-    static bool attr_set[64] = {false};   // the attribute is per device
-    if (!attr_set[ctx->device & 63]) {
+    static std::atomic<bool> attr_set[64];   // the attribute is per device
+    if (!attr_set[ctx->device & 63].load()) {
         ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(mean_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM));
-        attr_set[ctx->device & 63] = true;
+        attr_set[ctx->device & 63].store(true);
     }
     const int grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
     mean_grad_kernel<<<grid, MG_THREADS, MG_SMEM, st>>>(tmX, tmD, tmS, a);
@@ -1104,10 +1105,10 @@ int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
     a.n = n; a.S = S; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
     if (S && !accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
-    static bool attr_set[64] = {false};   // the attribute is per device
-    if (!attr_set[ctx->device & 63]) {
+    static std::atomic<bool> attr_set[64];   // the attribute is per device
+    if (!attr_set[ctx->device & 63].load()) {
         ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(direct_sqnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_SMEM));
-        attr_set[ctx->device & 63] = true;
+        attr_set[ctx->device & 63].store(true);
     }
     const int grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
     direct_sqnorm_kernel<<<grid, DR_THREADS, DR_SMEM, st>>>(tmX, tmD, tmS, a);

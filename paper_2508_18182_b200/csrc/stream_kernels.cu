@@ -7,6 +7,7 @@
 // arithmetic per byte is far below the machine balance, so grids are sized to
 // a multiple of the SM count and the only tuning that matters is bytes in
 // flight per SM.
+#include <mutex>
 #include <type_traits>
 
 #include "common.cuh"
@@ -390,15 +391,20 @@ static int launch_nt(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
     auto kern = norm_test_kernel<RB, VEC, BF16>;
     if (smem > 48 * 1024) ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // resident blocks per SM for this instantiation and shared-memory size (asked once)
+    static std::mutex cache_mutex;            // contexts on different host threads share these statics
     static size_t cached_smem = ~(size_t)0;
     static int cached_per_sm = 0;
-    if (cached_smem != smem) {
-        int q = 0;
-        ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&q, kern, NT_THREADS, smem));
-        cached_per_sm = q;
-        cached_smem = smem;
+    int per_sm;
+    {
+        std::lock_guard<std::mutex> lock(cache_mutex);
+        if (cached_smem != smem) {
+            int q = 0;
+            ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&q, kern, NT_THREADS, smem));
+            cached_per_sm = q;
+            cached_smem = smem;
+        }
+        per_sm = cached_per_sm;
     }
-    const int per_sm = cached_per_sm;
     if (per_sm < 1) return ADLOCO_ERR_WORKSPACE;
     int64_t max_grid = (int64_t)ctx->sm_count * per_sm;
     if (max_grid > ctx->max_grid) max_grid = ctx->max_grid;
@@ -618,15 +624,20 @@ static int launch_ip_t(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
     auto kern = centred_dot_kernel<RB, VEC, BF16>;
     if (smem > 48 * 1024) ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // resident blocks per SM for this instantiation and shared-memory size (asked once)
+    static std::mutex cache_mutex;            // contexts on different host threads share these statics
     static size_t cached_smem = ~(size_t)0;
     static int cached_per_sm = 0;
-    if (cached_smem != smem) {
-        int q = 0;
-        ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&q, kern, NT_THREADS, smem));
-        cached_per_sm = q;
-        cached_smem = smem;
+    int per_sm;
+    {
+        std::lock_guard<std::mutex> lock(cache_mutex);
+        if (cached_smem != smem) {
+            int q = 0;
+            ADLOCO_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&q, kern, NT_THREADS, smem));
+            cached_per_sm = q;
+            cached_smem = smem;
+        }
+        per_sm = cached_per_sm;
     }
-    const int per_sm = cached_per_sm;
     if (per_sm < 1) return ADLOCO_ERR_WORKSPACE;
     int64_t max_grid = (int64_t)ctx->sm_count * per_sm;
     if (max_grid > ctx->max_grid) max_grid = ctx->max_grid;
@@ -779,11 +790,6 @@ constexpr int NA_MAX_DEVICES = 64;
 static void* g_noalloc_ptr[NA_MAX_DEVICES];   // device address of the array, per device; nullptr until set up
 static int g_noalloc_sms[NA_MAX_DEVICES];
 
-}  // namespace adloco
-
-#include <mutex>
-
-namespace adloco {
 static std::mutex g_noalloc_mutex;
 
 template <int RB, bool VEC>
@@ -989,9 +995,11 @@ __global__ void __launch_bounds__(256, KB == 8 ? 4 : 6) outer_step_kernel(const 
 template <typename Kern>
 static unsigned elementwise_grid(const adloco_ctx* ctx, Kern kern, int64_t nvec, int threads) {
     // resident blocks per SM, asked once per kernel
+    static std::mutex cache_mutex;
     static const void* seen[16];
     static int seen_per_sm[16];
     static int n_seen = 0;
+    std::lock_guard<std::mutex> lock(cache_mutex);
     int per_sm = 0;
     for (int k = 0; k < n_seen; ++k)
         if (seen[k] == reinterpret_cast<const void*>(kern)) per_sm = seen_per_sm[k];
