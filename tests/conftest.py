@@ -24,3 +24,19 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_built():
+    """GPU runs start from the in-tree libadloco.so; if it is absent or older than its
+    sources it is rebuilt here (nvcc is part of the image).  A failed build fails the run:
+    there is nothing to fall back to."""
+    try:
+        import torch
+        has_gpu = torch.cuda.is_available()
+    except Exception:
+        has_gpu = False
+    if has_gpu:
+        from paper_2508_18182_b200.build import build
+        build()
+    yield
