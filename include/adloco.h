@@ -59,7 +59,9 @@ enum {
     ADLOCO_FLAG_GROW = 1,       /* b_req > b_cur */
     ADLOCO_FLAG_ACCUMULATE = 2, /* switch mode: b_req > switch_n * b_max */
     ADLOCO_FLAG_UNDEFINED = 4,  /* batch_count - ddof <= 0: no variance; b_req = max(1, b_cur) */
-    ADLOCO_FLAG_ZERO_MEAN = 8   /* ||gbar||^2 == 0: stat = +inf, b_req = b_cap or INT64_MAX */
+    ADLOCO_FLAG_ZERO_MEAN = 8,  /* ||gbar||^2 == 0: stat = +inf, b_req = b_cap or INT64_MAX */
+    ADLOCO_FLAG_NONFINITE = 16  /* a sum is Inf or NaN (an overflowed gradient): variance = stat = 0
+                                   are placeholders, b_req = max(1, b_cur); checked before the others */
 };
 
 /* Parameters of the batch rule and of switch mode.
@@ -204,7 +206,8 @@ typedef struct {
 
 /* var_ip = Var_i <g_i, gbar>, stat_ip = var_ip / (theta^2 ||gbar||^4), b_ip = max(1, ceil(stat_ip));
  * var_orth = Var_i (g_i - (<g_i, gbar> / ||gbar||^2) gbar), stat_orth = var_orth / (nu^2 ||gbar||^2),
- * b_aug = max(b_ip, ceil(stat_orth)).  Flags GROW (b_aug > b_cur), UNDEFINED, ZERO_MEAN as for the norm test. */
+ * b_aug = max(b_ip, ceil(stat_orth)).  Flags GROW (b_aug > b_cur), UNDEFINED, ZERO_MEAN, NONFINITE as for the
+ * norm test. */
 typedef struct {
     double var_ip;
     double stat_ip;

@@ -21,7 +21,8 @@ choice):
     (1/(b - ddof)) * sum_i ||g_i - gbar||^2, ddof = 1 by default.
   * b_{k+1} = max(1, ceil(stat)); a zero mean gradient gives stat = +inf.
   * b - ddof <= 0 leaves the variance undefined: V = 0, stat = 0, the batch
-    stays at max(1, b_cur).
+    stays at max(1, b_cur).  The same holds when a sum is Inf or NaN (flag
+    NONFINITE), which is checked first.
   * OuterOpt is SGD with (optionally Nesterov) momentum, no dampening:
     v' = mu v + d, u = d + mu v' (Nesterov) or v' (heavy ball),
     theta' = theta - lr u, with d the mean over the K instances of
@@ -49,6 +50,7 @@ FLAG_GROW = 1
 FLAG_ACCUMULATE = 2
 FLAG_UNDEFINED = 4
 FLAG_ZERO_MEAN = 8
+FLAG_NONFINITE = 16
 
 INT64_MAX = (1 << 63) - 1
 
@@ -107,7 +109,12 @@ def decide(sum_sqnorm: float, mean_sqnorm: float, variance: float, b: int, *,
     if not (eta > 0.0 and math.isfinite(eta)):
         raise ValueError("eta must be positive and finite")
     r = NormTestResult(sum_sqnorm=sum_sqnorm, mean_sqnorm=mean_sqnorm, batch_count=b)
-    if b - ddof <= 0:
+    if not (math.isfinite(sum_sqnorm) and math.isfinite(mean_sqnorm) and math.isfinite(variance)):
+        # an Inf or NaN gradient entry leaves no statistic to test: the batch stays
+        r.flags |= FLAG_NONFINITE
+        r.variance, r.stat = 0.0, 0.0
+        r.b_req = max(1, b_cur)
+    elif b - ddof <= 0:
         r.flags |= FLAG_UNDEFINED
         r.variance, r.stat = 0.0, 0.0
         r.b_req = max(1, b_cur)
@@ -204,7 +211,10 @@ def inner_product_tests(G, *, theta: float, nu: float, ddof: int = 1, b_cur: int
     gbar = total / b
     N = float(np.dot(gbar, gbar))
     r = InnerProductResult(mean_sqnorm=N, batch_count=b)
-    if b - ddof <= 0:
+    if not math.isfinite(N):
+        r.flags |= FLAG_NONFINITE
+        r.b_ip = r.b_aug = max(1, b_cur)
+    elif b - ddof <= 0:
         r.flags |= FLAG_UNDEFINED
         r.b_ip = r.b_aug = max(1, b_cur)
     elif N == 0.0:
@@ -281,7 +291,9 @@ def vector_param_terms(D, X=None):
 def embedding_terms(ids, D, V: int):
     """Per-sample gradients of an embedding table E [V, d] looked up at every token:
     row v of sample i's gradient is the sum of delta_{i,t} over the tokens t with
-    ids[i, t] = v.  ids [B, T] integers in [0, V), D [B, T, d].
+    ids[i, t] = v.  ids [B, T] integers, D [B, T, d].  A token whose id lies
+    outside [0, V) (padding, an ignore marker) looks up no row of E, so it has no
+    term in any row's sum: it is dropped.
     Returns n_i = ||G_i||_F^2 and S = sum_i G_i ([V, d])."""
     ids = np.asarray(ids)
     B = ids.shape[0]
@@ -290,7 +302,8 @@ def embedding_terms(ids, D, V: int):
     S = np.zeros((V, d), dtype=np.float64)
     for i in range(B):
         G_i = np.zeros((V, d), dtype=np.float64)
-        np.add.at(G_i, ids[i], widen(D[i]))
+        inside = (ids[i] >= 0) & (ids[i] < V)
+        np.add.at(G_i, ids[i][inside], widen(D[i])[inside])
         n[i] = float(np.sum(G_i * G_i))
         S += G_i
     return n, S

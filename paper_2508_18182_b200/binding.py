@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libadloco.so")
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
 F32, BF16 = 0, 1
-FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN = 1, 2, 4, 8
+FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN, FLAG_NONFINITE = 1, 2, 4, 8, 16
 
 # every symbol that include/adloco.h declares
 EXPORTS = (
@@ -335,6 +335,8 @@ def norm_test_noalloc(G, params: TestParams, result_dev, result_host, *, per_sam
     (pinned host) are uint8 tensors of at least sizeof(TestResult) bytes that the
     caller owns.  Returns the TestResult after synchronising the stream."""
     lib = load_library()
+    if G.dtype != torch.float32 or G.stride(1) != 1:
+        raise AdlocoError(ERR_UNSUPPORTED, "adloco_norm_test_noalloc takes float32 rows with contiguous columns")
     B, P = G.shape
     stride = G.stride(0) if B > 1 else max(G.stride(0), P)
     rc = lib.adloco_norm_test_noalloc(_ptr(G), B, P, stride, C.byref(params), _ptr(per_sample_sqnorm),

@@ -260,6 +260,7 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 struct EmbedArgs {
     GramArgs g;          // B, T, d_out = embedding width, item bookkeeping, n, status, wait bound
     const int* ids;      // [B, T]
+    int V;               // rows of the table: ids outside [0, V) belong to no row and match nothing
 };
 
 __global__ void __launch_bounds__(GR_THREADS, 1)
@@ -369,10 +370,12 @@ embed_gram_kernel(const __grid_constant__ CUtensorMap tmD, const EmbedArgs ea) {
         for (int item = blockIdx.x; item < a.total_items; item += gridDim.x, ++n_item) {
             int i, ti, c0, ncb;
             gram_decode(item, a, i, ti, c0, ncb);
-            // ids of this thread's row and of the columns it will visit; tokens beyond T never match
+            // ids of this thread's row and of the columns it will visit; tokens beyond T and ids
+            // outside the table (padding, ignore markers) get two different sentinels: they match nothing
             const int* ids_i = ea.ids + (int64_t)i * a.T;
             const int t_row = ti * GR_TILE + (int)q * 32 + lane;
-            const int id_row = t_row < a.T ? __ldg(ids_i + t_row) : -1;
+            int id_row = t_row < a.T ? __ldg(ids_i + t_row) : -1;
+            if (id_row < 0 || id_row >= ea.V) id_row = -1;
             const uint32_t buf = n_item & 1, use = n_item >> 1;
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abortp, a.wait_ns))) break;
             tc_fence_after();
@@ -385,7 +388,8 @@ embed_gram_kernel(const __grid_constant__ CUtensorMap tmD, const EmbedArgs ea) {
                 uint32_t d[32];
                 tmem_ld32(taddr + col, d);
                 const int t_col = c0 * GR_TILE + col + lane;                 // lane l holds the id of column col + l
-                const int id_col = t_col < a.T ? __ldg(ids_i + t_col) : -2;
+                int id_col = t_col < a.T ? __ldg(ids_i + t_col) : -2;
+                if (id_col < 0 || id_col >= ea.V) id_col = -2;
                 tmem_ld_wait();
                 float part = 0.f;
 #pragma unroll
@@ -1025,6 +1029,7 @@ int launch_embedding(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, 
     a.total_items = (int)((fulls + halves) * B);
     a.n = n; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     ea.ids = ids;
+    ea.V = (int)V;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
     static std::atomic<bool> attr_set[64];   // the attribute is per device
     if (!attr_set[ctx->device & 63].load()) {

@@ -145,7 +145,14 @@ __device__ void decide_device(const adloco_test_sums& s, const adloco_test_param
     r.flags = 0;
     r.device_status = s.device_status;
     const int64_t i64max = 0x7fffffffffffffffLL;
-    if (b - p.ddof <= 0) {
+    // an overflowed or NaN gradient anywhere poisons every sum: no statistic, the batch stays
+    const bool finite = isfinite(s.sum_sqnorm) && isfinite(s.sum_sq_gsum) && (!s.has_centred || isfinite(s.centred_ss));
+    if (!finite) {
+        r.flags |= ADLOCO_FLAG_NONFINITE;
+        r.variance = 0.0;
+        r.stat = 0.0;
+        r.b_req = p.b_cur > 1 ? p.b_cur : 1;
+    } else if (b - p.ddof <= 0) {
         r.flags |= ADLOCO_FLAG_UNDEFINED;
         r.variance = 0.0;
         r.stat = 0.0;
@@ -359,6 +366,8 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
         } else {  // NT_MICRO: rows are appended
             const double cp = (double)s.batch_count, bb = (double)B;
             s.centred_ss += css + (cp > 0.0 ? (cp * bb / (cp + bb)) * chan : 0.0);
+            // the centred sum stays valid while every micro-batch so far came materialised
+            if (cp == 0.0) s.has_centred = 1;
             s.sum_sqnorm += Q;
             s.sum_sq_gsum = sumsq;  // ||S||^2 of the updated sum buffer
             s.batch_count += B;
@@ -485,7 +494,12 @@ __device__ void ip_decide_device(double sum_d2, double sum_d, const adloco_test_
     r.flags = 0;
     r.device_status = s.device_status;
     r.var_ip = r.stat_ip = r.var_orth = r.stat_orth = 0.0;
-    if (b - p.ddof <= 0) {
+    const bool finite = isfinite(sum_d2) && isfinite(sum_d) && isfinite(s.sum_sqnorm) && isfinite(s.sum_sq_gsum) &&
+                        (!s.has_centred || isfinite(s.centred_ss));
+    if (!finite) {
+        r.flags |= ADLOCO_FLAG_NONFINITE;
+        r.b_ip = r.b_aug = p.b_cur > 1 ? p.b_cur : 1;
+    } else if (b - p.ddof <= 0) {
         r.flags |= ADLOCO_FLAG_UNDEFINED;
         r.b_ip = r.b_aug = p.b_cur > 1 ? p.b_cur : 1;
     } else if (N == 0.0) {

@@ -70,3 +70,22 @@ def test_exact_on_integers_and_special_id_patterns(ctx):
     with pytest.raises(A.AdlocoError) as e:
         ctx.embedding_sqnorm(ids, D[:, :, :12].contiguous(), 9, n)
     assert e.value.status == A.ERR_UNSUPPORTED and ctx.launch_count == before
+
+
+def test_ids_outside_the_table_are_dropped_from_norms_and_sum(ctx):
+    """Padding / ignore ids (-100, ids >= V) look up no row: they add nothing to n_i or S, and two
+    tokens that share such an id do not pair up in the masked Gram sum."""
+    B, T, d, V = 4, 300, 64, 11
+    _, D = W.small_integer_layer(B, T, 8, d, seed=8, device=DEV)
+    ids = _ids(B, T, V, seed=2)
+    ids[0, 5:90] = -100                     # a run of one repeated padding id, crossing a 128-token block
+    ids[1, ::3] = V                         # first id past the table
+    ids[2, 200:] = V + 1000
+    ids[3, :] = -1                          # a sample with no token inside the table
+    n = torch.full((B,), -1.0, device=DEV)
+    S = torch.full((V, d), -1.0, device=DEV)
+    ctx.embedding_sqnorm(ids, D, V, n, grad_sum=S)
+    torch.cuda.synchronize()
+    n_ref, S_ref = O.embedding_terms(ids.cpu().numpy(), W.to_numpy(D), V)
+    assert np.array_equal(n.cpu().numpy().astype(np.float64), n_ref) and n_ref[3] == 0.0
+    assert np.array_equal(S.cpu().numpy().astype(np.float64), S_ref)

@@ -109,46 +109,52 @@ def test_config3_gram_layer_full_size(ctx):
 
 # ---------------------------------------------------------------- config 4
 def test_config4_whole_model_switch_mode_full_size(ctx):
-    """12 blocks x 4 linear layers, batch 128 as 4 accumulated micro-batches of 32.
-    The GPU runs everything; the oracle checks sampled (layer, micro-batch) units
-    (per-sample norms of two samples, three rows of the gradient sum) and the
-    closed form of the statistic for pure-noise gradients."""
+    """12 blocks x 4 linear layers, batch 128 as 4 accumulated micro-batches of 32, by both routes
+    (the Gram identity, and whatever route AUTO picks: the direct one for these shapes).  The oracle
+    runs the whole model once, streamed layer by layer and micro-batch by micro-batch (explicit
+    per-sample gradients in fp64; about a minute of host BLAS), and every output is compared: the
+    128 per-sample norms, each layer's gradient sum element by element, ||S_l||^2 per layer, and the
+    statistic, decision and switch plan."""
     shapes = list(W.GPT2_SMALL_BLOCK_LINEARS) * 12
     n_micro, b, T = 4, 32, 1024
-    sums = [torch.empty(do, di, device=DEV) for di, do in shapes]
-    acc = A.Accumulator(ctx, sums)
-    acc.reset()
-    sampled = {(0, 0), (13, 2), (47, 3), (22, 1)}        # (layer, micro-batch)
-    rows = (0, 5, 767)
-    row_ref = {l: np.zeros((len(rows), shapes[l][0])) for l, _ in sampled}
-    n_mb = torch.zeros(b, device=DEV)
-    n_layer = torch.zeros(b, device=DEV)
+    routes = ("gram", "auto")
+    sums = {m: [torch.empty(do, di, device=DEV) for di, do in shapes] for m in routes}
+    accs = {m: A.Accumulator(ctx, sums[m]) for m in routes}
+    n_mb = {m: torch.zeros(b, device=DEV) for m in routes}
+    n_all = {m: torch.zeros(n_micro * b, device=DEV) for m in routes}
+    for m in routes:
+        accs[m].reset()
+    n_ref = np.zeros(n_micro * b)
+    S_ref = [np.zeros((do, di)) for di, do in shapes]
     for j in range(n_micro):
         for l, (di, do) in enumerate(shapes):
             X, D = W.linear_layer(b, T, di, do, seed=100000 + 100 * l + j, device=DEV)
-            ctx.gram_sqnorm(X, D, n_mb, accumulate_norms=(l > 0), grad_sum=sums[l], accumulate_sum=True)
-            if (l, j) in sampled:
-                ctx.gram_sqnorm(X, D, n_layer)            # this layer's norms alone
-                torch.cuda.synchronize()
-                for i in (0, b - 1):
-                    G_i = O.per_sample_weight_grad(W.to_numpy(X[i]), W.to_numpy(D[i]))
-                    assert rel_close(float(n_layer[i]), float((G_i ** 2).sum()), TOL_BF16), (l, j, i)
-            if any(l == ls for ls, _ in sampled):
-                Xd = X.reshape(-1, di).double()
-                for k, o in enumerate(rows):                 # S_l[o, :] += Delta[:, o]^T X, on the host in fp64
-                    row_ref[l][k] += (D.reshape(-1, do)[:, o].double().cpu().numpy() @ Xd.cpu().numpy())
+            for m in routes:
+                ctx.linear_sqnorm(X, D, n_mb[m], accumulate_norms=(l > 0), grad_sum=sums[m][l], accumulate_sum=True,
+                                  method=m)
+            n_l, S_l = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))     # overlaps the GPU work
+            n_ref[j * b:(j + 1) * b] += n_l
+            S_ref[l] += S_l
             del X, D
-        acc.accumulate(per_sample_sqnorm=n_mb)
+        for m in routes:
+            accs[m].accumulate(per_sample_sqnorm=n_mb[m])
+            n_all[m][j * b:(j + 1) * b] = n_mb[m]
     p = A.make_params(0.5, b_cur=128, b_max=32)
-    r = acc.finalize(p)
-    for l, ref in row_ref.items():
-        got = sums[l][list(rows)].cpu().numpy()
-        assert np.allclose(got, ref, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(ref).max() * 0.05), l
-    # pure-noise gradients: stat ~ B / eta^2 = 512, relative sd ~ sqrt(2 / P_total) (tiny)
-    assert r.batch_count == 128 and abs(r.stat - 512.0) < 0.01 * 512.0, r.stat
-    assert r.flags & A.FLAG_ACCUMULATE and r.flags & A.FLAG_GROW
-    assert abs(r.b_req - 512) <= 6 and r.b_micro == 32 and abs(r.accum_steps - 16) <= 1
-    acc.close()
+    ora = O.norm_test_from_sums(n_ref, S_ref, n_micro * b, eta=0.5, b_cur=128, b_max=32)
+    kappa = ora.sum_sqnorm / (ora.variance * (n_micro * b - 1))
+    for m in routes:
+        r = accs[m].finalize(p)
+        assert ctx.device_status() == 0
+        assert np.allclose(n_all[m].cpu().numpy(), n_ref, rtol=TOL_BF16, atol=0), m
+        for l in range(len(shapes)):
+            got = sums[m][l].cpu().numpy().astype(np.float64)
+            assert np.allclose(got, S_ref[l], rtol=TOL_BF16, atol=TOL_BF16 * np.abs(S_ref[l]).max() * 0.05), (m, l)
+            assert rel_close(float((got ** 2).sum()), float((S_ref[l] ** 2).sum()), TOL_BF16), (m, l)
+        assert_test_result(r, ora, p, TOL_BF16, stat_tol=TOL_BF16 * max(1.0, kappa), what=f"config 4 {m}")
+        assert r.batch_count == 128 and r.flags & A.FLAG_ACCUMULATE and r.flags & A.FLAG_GROW and r.b_micro == 32
+        # pure-noise gradients: stat ~ B / eta^2 = 512
+        assert abs(r.stat - 512.0) < 0.01 * 512.0, r.stat
+        accs[m].close()
 
 
 # ---------------------------------------------------------------- config 5

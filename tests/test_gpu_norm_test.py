@@ -218,6 +218,68 @@ def test_accumulated_test_matches_one_shot_oracle(ctx, n_micro, b, P, sigma, sca
     acc.close()
 
 
+@pytest.mark.parametrize("sigma", [1e-3, 3e-5])
+def test_accumulated_variance_keeps_its_digits_when_the_mean_dominates(ctx, sigma):
+    """Mean far above the noise: Q - b N would cancel 6 to 9 digits (sum_i n_i / ((b-1) V) ~ 1e6 .. 1e9).
+    The materialised accumulation keeps the column-centred sum of squares across micro-batches, so
+    the accumulated variance must match the one-shot test and the oracle as if nothing cancelled."""
+    n_micro, b, P = 6, 16, 40000
+    mbs = W.micro_batches(n_micro, b, P, sigma=sigma, mean_scale="raw", seed=77, device=DEV)
+    S = torch.empty(P, device=DEV)
+    acc = A.Accumulator(ctx, [S])
+    acc.reset()
+    for m in mbs:
+        acc.accumulate(m)
+    p = A.make_params(0.5, b_cur=n_micro * b, b_max=b)
+    r = acc.finalize(p)
+    sums = ctx.read_sums()
+    assert sums.has_centred == 1 and sums.batch_count == n_micro * b
+    ora = O.accumulated_norm_test([W.to_numpy(m) for m in mbs], eta=0.5, b_cur=n_micro * b, b_max=b)
+    assert ora.sum_sqnorm / (ora.variance * (n_micro * b - 1)) > 1e5
+    assert_test_result(r, ora, p, TOL_F32, what="signal-dominated accumulation")
+    one = ctx.norm_test(torch.cat(mbs), p)
+    assert rel_close(one.variance, r.variance, TOL_F32) and rel_close(one.stat, r.stat, TOL_F32)
+    # a form-(b) call in between drops the centred sum for good: the identity takes over
+    acc.reset()
+    acc.accumulate(mbs[0])
+    n1 = torch.zeros(b, device=DEV)
+    ctx.norm_test(mbs[1], p, per_sample_sqnorm=n1)
+    S += mbs[1].sum(0)
+    acc.accumulate(per_sample_sqnorm=n1)
+    acc.finalize(p)
+    assert ctx.read_sums().has_centred == 0
+    acc.close()
+
+
+@pytest.mark.parametrize("bad", [float("inf"), float("nan"), 3e38])
+def test_nonfinite_gradients_raise_the_flag_and_keep_the_batch(ctx, bad):
+    """One Inf / NaN entry (or one whose square overflows fp32) poisons the sums: the result carries
+    NONFINITE, the batch stays at b_cur and the switch plan is that of b_cur -- no huge request."""
+    G = W.per_sample_grads(8, 5000, seed=6, device=DEV)
+    G[3, 1234] = bad
+    p = A.make_params(0.5, b_cur=8, b_max=32)
+    r = ctx.norm_test(G, p)
+    assert r.flags == A.FLAG_NONFINITE and r.b_req == 8 and r.stat == 0.0 and r.variance == 0.0
+    assert (r.accum_steps, r.b_micro) == (1, 8)
+    if bad != 3e38:
+        Gn = W.to_numpy(G)
+        assert_test_result(r, O.norm_test(Gn, eta=0.5, b_cur=8, b_max=32), p, TOL_F32, what="non-finite")
+        S = torch.empty(5000, device=DEV)
+        ctx.norm_test(G, p, grad_sum=S)
+        ri = ctx.inner_product_test(G, S, theta=0.1, nu=0.3, b_cur=8)
+        assert ri.flags == A.FLAG_NONFINITE and ri.b_ip == ri.b_aug == 8
+    # the accumulator reports it too
+    S = torch.empty(5000, device=DEV)
+    acc = A.Accumulator(ctx, [S])
+    acc.reset()
+    acc.accumulate(G)
+    ra = acc.finalize(p)
+    assert ra.flags == A.FLAG_NONFINITE and ra.b_req == 8
+    acc.close()
+    G[3, 1234] = 0.0
+    assert ctx.norm_test(G, p).flags & A.FLAG_NONFINITE == 0
+
+
 def test_accumulate_from_given_norms_uses_the_identity(ctx):
     # form (b): the caller adds the gradient sums itself and hands over n_i
     mbs = W.micro_batches(3, 8, 5000, sigma=1.0, seed=3, device=DEV)

@@ -253,6 +253,27 @@ def pin_embedding_terms(O):
     n_e, S_e = O.embedding_terms(np.full((3, 7), 2), Dn, 4)
     n_b, S_b = O.vector_param_terms(Dn)
     assert np.array_equal(n_e, n_b) and np.array_equal(S_e[2], S_b) and not S_e[[0, 1, 3]].any()
+    # tokens whose id names no row of the table (padding such as -100, ids >= V) have no gradient:
+    # brute force over the tokens that remain; two padding tokens must not pair up with each other
+    pad = ids.copy()
+    pad[0, 1] = pad[0, 4] = -100
+    pad[1, 0] = pad[1, 6] = V
+    pad[2, 3] = V + 7
+    n_p, S_p = O.embedding_terms(pad, Dn, V)
+    S_ref = [[0] * 8 for _ in range(V)]
+    for i in range(3):
+        G = [[0] * 8 for _ in range(V)]
+        for t in range(7):
+            if 0 <= int(pad[i, t]) < V:
+                for j in range(8):
+                    G[int(pad[i, t])][j] += int(Di[i][t][j])
+        assert n_p[i] == float(sum(x * x for row in G for x in row))
+        for v in range(V):
+            for j in range(8):
+                S_ref[v][j] += G[v][j]
+    assert S_p.tolist() == [[float(x) for x in row] for row in S_ref]
+    n_none, S_none = O.embedding_terms(np.full((3, 7), -1), Dn, V)
+    assert not n_none.any() and not S_none.any()
 
 
 def pin_layers_test_two_routes(O):
@@ -394,6 +415,29 @@ def pin_inner_product_tests(O):
         O.inner_product_tests(G, theta=0.0, nu=0.3)
 
 
+def pin_nonfinite_sums_leave_the_batch_alone(O):
+    # an Inf or NaN anywhere leaves no statistic: flag 16, V = stat = 0, b stays at max(1, b_cur), no NaN in the plan
+    for bad in (math.inf, -math.inf, math.nan):
+        for args in ((bad, 1.0, 1.0), (10.0, bad, 1.0), (10.0, 1.0, bad)):
+            r = O.decide(*args, 8, eta=0.5, b_cur=6, b_max=4)
+            assert r.flags == O.FLAG_NONFINITE and r.b_req == 6 and r.stat == 0.0 and r.variance == 0.0
+            assert (r.accum_steps, r.b_micro) == (1, 4)
+    assert O.decide(math.nan, 1.0, 1.0, 1, eta=0.5, b_cur=0).b_req == 1        # checked before UNDEFINED
+    assert O.decide(math.nan, 1.0, 1.0, 8, eta=0.5, b_cur=3, b_max=1).flags == O.FLAG_NONFINITE | O.FLAG_ACCUMULATE
+    G = W.to_numpy(W.per_sample_grads(4, 64, seed=3)).copy()
+    for bad in (np.float32(np.inf), np.float32(np.nan), np.float32(3e38)):     # 3e38 squared overflows only in fp32
+        H = G.copy()
+        H[2, 5] = bad
+        r = O.norm_test(H, eta=0.5, b_cur=4, b_max=32)
+        if np.isfinite(bad):
+            assert r.flags & O.FLAG_NONFINITE == 0 and math.isfinite(r.stat)   # fp64 holds 9e76
+        else:
+            assert r.flags & O.FLAG_NONFINITE and r.b_req == 4
+            ip = O.inner_product_tests(H, theta=0.1, nu=0.3, b_cur=4)
+            assert ip.flags & O.FLAG_NONFINITE and ip.b_ip == ip.b_aug == 4
+    assert O.decide(10.0, 1.0, 1.0, 8, eta=0.5).flags & O.FLAG_NONFINITE == 0
+
+
 PINS = [v for k, v in sorted(globals().items()) if k.startswith("pin_")]
 
 
@@ -429,7 +473,11 @@ MUTANTS = [
     ("merge takes the largest", "order = sorted(range(k), key=lambda i: (b_req[i], i))",
      "order = sorted(range(k), key=lambda i: (-b_req[i], i))"),
     ("merge unweighted", "x += float(b) * widen(p)", "x += widen(p)"),
-    ("embedding rows overwritten instead of summed", "np.add.at(G_i, ids[i], widen(D[i]))", "G_i[ids[i]] = widen(D[i])"),
+    ("embedding rows overwritten instead of summed", "np.add.at(G_i, ids[i][inside], widen(D[i])[inside])",
+     "G_i[ids[i][inside]] = widen(D[i])[inside]"),
+    ("padding ids wrap around into the table", "inside = (ids[i] >= 0) & (ids[i] < V)", "inside = ids[i] < V"),
+    ("non-finite sums pass through", "if not (math.isfinite(sum_sqnorm) and math.isfinite(mean_sqnorm) and math.isfinite(variance)):",
+     "if False:"),
     ("vector parameter summed over features", "g = (d * widen(X[i])).sum(axis=0) if X is not None else d.sum(axis=0)",
      "g = (d * widen(X[i])).sum(axis=1) if X is not None else d.sum(axis=1)"),
     ("gain gradient without the input", "g = (d * widen(X[i])).sum(axis=0) if X is not None else d.sum(axis=0)",
