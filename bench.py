@@ -1,16 +1,24 @@
 #!/usr/bin/env python
 """Benchmark of the AdLoCo hot path on B200.
 
-One step = one pass of the whole path over one batch of synthetic input:
+One step = one pass of the whole path over one batch of synthetic input, at the
+sizes of the workload configurations:
   1. norm test on materialised per-sample gradients (B=64, P=2^24 fp32), with the
      batch decision for eta in {0.1, 0.5, 1.0} from one pass over the gradients;
   2. outer step over K=8 bf16 instances of a 124M-parameter vector (fp32 global
      parameters and momentum, lr 0.7, Nesterov momentum 0.9), in place;
   3. Gram-identity per-sample norms + mean-gradient GEMM for one linear layer
      (X bf16 [32,1024,768], Delta bf16 [32,1024,3072]), accumulated into a
-     switch-mode accumulator and finalised into one test.
-The headline value is the HBM throughput of the streaming part (1 + 2):
-algorithmic bytes / device time.  The tensor-core part is reported beside it.
+     switch-mode accumulator and finalised into one test;
+  4. the whole-model test in switch mode: 12 blocks x 4 linear layers x 4
+     micro-batches of 32 sequences through adloco_linear_sqnorm (automatic
+     route), per-sample norms accumulated over layers, gradient sums over
+     micro-batches, one test at the end;
+  5. outer step over K=4 bf16 instances of a 1.3B-parameter vector, in place;
+  6. the norm test over 8 accumulated micro-batches of 32 x 2^22 fp32 gradients.
+The headline value is the HBM throughput of the streaming sections (1, 2, 5, 6):
+algorithmic bytes / device time.  The tensor-core sections (3, 4) are reported
+beside it; the roofline entry is the dominant kernel of the step by time.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -43,14 +51,23 @@ NT_B, NT_P = 64, 1 << 24
 OUT_K, OUT_P = 8, W.GPT2_SMALL_P
 ETAS = (0.1, 0.5, 1.0)
 LR, MU = 0.7, 0.9
-# the tensor-core workload
+# the tensor-core workload: one linear layer (configs[2]) ...
 GR_B, GR_T, GR_DIN, GR_DOUT = 32, 1024, 768, 3072
+# ... the whole model in switch mode (configs[3]): 12 blocks x 4 linear layers, 4 micro-batches of 32
+C4_SHAPES = list(W.GPT2_SMALL_BLOCK_LINEARS) * 12
+C4_B, C4_MICRO = 32, 4
+# the large outer merge and the accumulated test (configs[4])
+C5_K, C5_P = 4, W.LARGE_P
+C5_B, C5_MICRO, C5_ACC_P = 32, 8, 1 << 22
 
 
 def algorithmic_bytes():
+    """Bytes each streaming section must move once (read + written), per step."""
     nt = 4 * NT_B * NT_P                               # every gradient element read once
     outer = (2 * OUT_K + 8) * OUT_P + 8 * OUT_P        # K bf16 instances + theta + v read; theta + v written
-    return nt, outer
+    outer5 = (2 * C5_K + 8) * C5_P + 8 * C5_P
+    acc5 = C5_MICRO * (4 * C5_B + 8) * C5_ACC_P        # micro-batch rows read + S read-modify-written
+    return {"nt2": nt, "os2": outer, "os5": outer5, "acc5": acc5}
 
 
 def gram_flops():
@@ -59,6 +76,13 @@ def gram_flops():
     executed = 2 * GR_B * tiles * 128 * 128 * (GR_DIN + GR_DOUT)  # at 128-token tile granularity
     mean_grad = 2 * GR_B * GR_T * GR_DIN * GR_DOUT
     return sym, executed, mean_grad
+
+
+def model_flops():
+    """Algorithmic flops of the whole-model test by the direct route: one GEMM
+    2 b T d_in d_out per (layer, micro-batch)."""
+    per_mb = sum(2 * C4_B * GR_T * di * do for di, do in C4_SHAPES)
+    return per_mb * C4_MICRO, len(C4_SHAPES) * C4_MICRO
 
 
 def reduce_max_over_ranks(values, device="cpu"):
@@ -150,35 +174,46 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------
 def oracle_sample_run(steps: int, warmup: int):
     """Times the oracle, as it stands, on a bounded sample of the streaming
-    workload: the norm test on B=64 x P=2^22 and the outer step on K=8 x P=2^23.
-    Returns (GB/s over the sample's algorithmic bytes, ms per step, threads)."""
-    import numpy as np
+    workload: the norm test on B=64 x P=2^22, the outer steps on K=8 x P=2^23 and
+    K=4 x P=2^23, and the accumulated test on 8 micro-batches of 32 x P=2^18.
+    Returns (GB/s over the sample's algorithmic bytes, ms per step, info)."""
     import oracle.adloco_oracle as O
     try:
         from threadpoolctl import threadpool_info
-        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        pool = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
-        threads = 1
-    sP, oP = 1 << 22, 1 << 23
+        pool = 1
+    sP, oP, aP = 1 << 22, 1 << 23, 1 << 18
     G = W.to_numpy(W.per_sample_grads(NT_B, sP, sigma=0.5, seed=1))
     theta, inst, mom = W.outer_state(OUT_K, oP, inst_dtype=torch.bfloat16, seed=2)
     th, v, ins = W.to_numpy(theta), W.to_numpy(mom), [W.to_numpy(t) for t in inst]
-    nbytes = 4 * NT_B * sP + (2 * OUT_K + 8) * oP + 8 * oP
+    theta5, inst5, mom5 = W.outer_state(C5_K, oP, inst_dtype=torch.bfloat16, seed=3)
+    th5, v5, ins5 = W.to_numpy(theta5), W.to_numpy(mom5), [W.to_numpy(t) for t in inst5]
+    mbs = [W.to_numpy(m) for m in W.micro_batches(C5_MICRO, C5_B, aP, sigma=1.0, mean_scale="raw", seed=4)]
+    nbytes = (4 * NT_B * sP + (2 * OUT_K + 16) * oP + (2 * C5_K + 16) * oP + C5_MICRO * (4 * C5_B + 8) * aP)
 
     def one():
         r = O.norm_test(G, eta=ETAS[0], b_cur=NT_B, b_max=32)
         for eta in ETAS[1:]:
             O.decide(r.sum_sqnorm, r.mean_sqnorm, r.variance, NT_B, eta=eta, b_cur=NT_B, b_max=32)
         O.outer_step(th, ins, v, lr=LR, momentum=MU, nesterov=True)
+        O.outer_step(th5, ins5, v5, lr=LR, momentum=MU, nesterov=True)
+        O.accumulated_norm_test(mbs, eta=0.5, b_cur=C5_B * C5_MICRO, b_max=32)
 
     for _ in range(warmup):
         one()
-    t0 = time.perf_counter()
+    t0, c0 = time.perf_counter(), time.process_time()
     for _ in range(steps):
         one()
-    dt = (time.perf_counter() - t0) / max(steps, 1)
-    sample = f"norm test B={NT_B} P=2^22 fp32 + outer step K={OUT_K} bf16 P=2^23 (1/4 resp. 1/15 of the workload)"
-    return nbytes / dt / 1e9, dt * 1e3, threads, sample
+    wall = time.perf_counter() - t0
+    cpu = time.process_time() - c0
+    dt = wall / max(steps, 1)
+    sample = (f"norm test B={NT_B} P=2^22 fp32 (1/4) + outer step K={OUT_K} bf16 P=2^23 (1/15) + outer step K={C5_K} bf16 "
+              f"P=2^23 (1/155) + accumulated test {C5_MICRO} x {C5_B} x 2^18 fp32 (1/16); the tensor-core part is not sampled")
+    # cores actually busy = CPU time of all threads of this process / wall time
+    info = {"cores": round(max(cpu / wall, 1.0), 2), "blas_pool_threads": pool, "sample": sample,
+            "cores_note": "process CPU time / wall time: the elementwise passes run on one thread, BLAS dot products on the pool"}
+    return nbytes / dt / 1e9, dt * 1e3, info
 
 
 def run_reference(args, rank):
@@ -186,13 +221,14 @@ def run_reference(args, rank):
         return
     steps = max(1, min(args.steps, 5))
     warm = max(1, min(args.warmup, 2))
-    gbs, ms, threads, sample = oracle_sample_run(steps, warm)
+    gbs, ms, info = oracle_sample_run(steps, warm)
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
         "config": workload_config(),
-        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": info["cores"], "kind": "oracle", "sample": info["sample"],
+                         "blas_pool_threads": info["blas_pool_threads"], "cores_note": info["cores_note"]},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -201,19 +237,29 @@ def run_reference(args, rank):
 
 def workload_config():
     if NT_P != 1 << 24:
-        return {"workload": f"profiling case: norm test B={NT_B} P={NT_P}, outer step K={OUT_K} P={OUT_P}, "
-                            f"Gram layer B={GR_B}", "l2": "inputs larger than L2 except the Gram layer",
-                "parallelism": "replicas"}
-    return {"workload": "configs[1] streaming scale-up: norm test B=64 P=16,777,216 fp32 (eta 0.1/0.5/1.0) + "
-                        "outer step K=8 bf16 P=124,439,808 (fp32 theta and momentum, lr 0.7, Nesterov 0.9); "
-                        "plus configs[2] Gram layer B=32 T=1024 768->3072 bf16 for the tensor-core figure",
-            "l2": "inputs larger than L2 (4.3 GB + 4.0 GB + 0.25 GB per step), no flush needed",
+        return {"workload": f"profiling case: norm test B={NT_B} P={NT_P}, outer step K={OUT_K} P={OUT_P}, Gram layer B={GR_B}, "
+                            f"{len(C4_SHAPES)} layers x {C4_MICRO} micro-batches by the automatic route, outer step K={C5_K} P={C5_P}, "
+                            f"accumulated test {C5_MICRO} x {C5_B} x {C5_ACC_P}",
+                "l2": "inputs larger than L2 except the single layers", "parallelism": "replicas"}
+    return {"workload": "configs[4] large outer merge + accumulated test: outer step K=4 bf16 P=1,300,000,000 (fp32 theta and "
+                        "momentum, lr 0.7, Nesterov 0.9, in place) and the norm test over 8 accumulated micro-batches of "
+                        "32 x 4,194,304 fp32; configs[3] whole-model switch mode: 12 blocks x 4 linear layers "
+                        "(768->2304, 768->768, 768->3072, 3072->768; T=1024 bf16) x 4 micro-batches of 32 through "
+                        "adloco_linear_sqnorm(auto), accumulated and tested once; configs[1] streaming scale-up: norm test "
+                        "B=64 P=16,777,216 fp32 (eta 0.1/0.5/1.0) + outer step K=8 bf16 P=124,439,808; configs[2] Gram layer "
+                        "B=32 T=1024 768->3072 bf16 (Gram identity + mean-gradient GEMM). value = bytes of the four streaming "
+                        "sections / their device time; the tensor-core sections are reported in roofline and kernels",
+            "l2": "inputs larger than L2 (72 GB resident; every section streams more than 126 MB except the single layers, "
+                  "whose operands are evicted by the 30 GB that pass between two visits), no flush needed",
             "parallelism": "replicas (no exchange step on the path)"}
 
 
 # ------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------
+SECTIONS = ("nt2", "os2", "gram3", "model4", "fin4", "os5", "acc5")
+
+
 def run_ours(args, rank, world, local_rank):
     from paper_2508_18182_b200 import binding as A
     from paper_2508_18182_b200.build import build
@@ -225,7 +271,7 @@ def run_ours(args, rank, world, local_rank):
     dev = torch.device("cuda", local_rank)
     ctx = A.Context(local_rank)
 
-    # ---- resident inputs
+    # ---- resident inputs (about 72 GB at full size)
     G = W.per_sample_grads(NT_B, NT_P, sigma=0.5, seed=10 + rank, device=dev)
     theta, inst, mom = W.outer_state(OUT_K, OUT_P, inst_dtype=torch.bfloat16, seed=20 + rank, device=dev)
     X, D = W.linear_layer(GR_B, GR_T, GR_DIN, GR_DOUT, seed=30 + rank, device=dev)
@@ -234,30 +280,64 @@ def run_ours(args, rank, world, local_rank):
     acc = A.Accumulator(ctx, [S_layer])
     params = [A.make_params(eta, b_cur=NT_B, b_max=32) for eta in ETAS]
     gparams = A.make_params(0.5, b_cur=GR_B, b_max=32)
+    # whole model: every (micro-batch, layer) pair of operands is resident
+    data4 = [[W.linear_layer(C4_B, GR_T, di, do, seed=1000 * j + l + 7 * rank, device=dev)
+              for l, (di, do) in enumerate(C4_SHAPES)] for j in range(C4_MICRO)]
+    sums4 = [torch.zeros(do, di, device=dev) for di, do in C4_SHAPES]
+    acc4 = A.Accumulator(ctx, sums4)
+    n_mb = torch.zeros(C4_B, device=dev)
+    p4 = A.make_params(0.5, b_cur=C4_B * C4_MICRO, b_max=32)
+    # large outer merge, accumulated test
+    theta5, inst5, mom5 = W.outer_state(C5_K, C5_P, inst_dtype=torch.bfloat16, seed=50 + rank, device=dev)
+    mbs5 = W.micro_batches(C5_MICRO, C5_B, C5_ACC_P, sigma=1.0, mean_scale="raw", seed=60 + rank, device=dev)
+    S5 = torch.zeros(C5_ACC_P, device=dev)
+    acc5 = A.Accumulator(ctx, [S5])
+    p5 = A.make_params(0.5, b_cur=C5_B * C5_MICRO, b_max=32)
     stream = torch.cuda.current_stream()
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
-    def step(marks=None):
-        if marks is not None:
-            marks["nt0"].record(stream)
+    def step(m=None):
+        def mark(name):
+            if m is not None:
+                e = ev()
+                e.record(stream)
+                m.append((name, e))
+        mark("begin")
+        # configs[1]: norm test with the eta sweep, outer step
         ctx.norm_test(G, params[0], sync=False)
-        if marks is not None:
-            marks["nt1"].record(stream)
         for p in params[1:]:
             ctx.test_decide(p, sync=False)
-        if marks is not None:
-            marks["os0"].record(stream)
+        mark("nt2")
         ctx.outer_step(inst, theta, mom, lr=LR, momentum=MU, nesterov=True)
-        if marks is not None:
-            marks["os1"].record(stream)
+        mark("os2")
+        # configs[2]: one layer by the Gram identity + mean-gradient GEMM, accumulated and tested
         acc.reset()
         ctx.gram_sqnorm(X, D, n_layer, grad_sum=S_layer, accumulate_sum=True)
         acc.accumulate(per_sample_sqnorm=n_layer)
         acc.finalize(gparams, sync=False)
-        if marks is not None:
-            marks["gr1"].record(stream)
+        mark("gram3")
+        # configs[3]: whole model, 4 micro-batches x 48 layers, one test
+        acc4.reset()
+        mark("fin4")
+        for j in range(C4_MICRO):
+            for l, (Xl, Dl) in enumerate(data4[j]):
+                ctx.linear_sqnorm(Xl, Dl, n_mb, accumulate_norms=(l > 0), grad_sum=sums4[l], accumulate_sum=True,
+                                  method="auto")
+            mark("model4")
+            acc4.accumulate(per_sample_sqnorm=n_mb)
+            if j == C4_MICRO - 1:
+                acc4.finalize(p4, sync=False)
+            mark("fin4")
+        # configs[4]: large outer merge, accumulated norm test
+        ctx.outer_step(inst5, theta5, mom5, lr=LR, momentum=MU, nesterov=True)
+        mark("os5")
+        acc5.reset()
+        for mb in mbs5:
+            acc5.accumulate(mb)
+        acc5.finalize(p5, sync=False)
+        mark("acc5")
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -269,7 +349,7 @@ def run_ours(args, rank, world, local_rank):
         dist.barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    marks = [{k: ev() for k in ("nt0", "nt1", "os0", "os1", "gr1")} for _ in range(args.steps)]
+    marks = [[] for _ in range(args.steps)]
     launches0 = ctx.launch_count
     torch.cuda.synchronize()
     t_begin, t_end = ev(), ev()
@@ -283,20 +363,23 @@ def run_ours(args, rank, world, local_rank):
         dist.barrier()
     clocks = sampler.stop()
     launches = ctx.launch_count - launches0
-    last = ctx._read_result()
+    res5 = ctx._read_result()
 
     total_ms = t_begin.elapsed_time(t_end)
-    nt_ms = sum(m["nt0"].elapsed_time(m["nt1"]) for m in marks) / args.steps
-    os_ms = sum(m["os0"].elapsed_time(m["os1"]) for m in marks) / args.steps
-    stream_ms = sum(m["nt0"].elapsed_time(m["os1"]) for m in marks) / args.steps
-    gram_ms = sum(m["os1"].elapsed_time(m["gr1"]) for m in marks) / args.steps
-    total_ms, stream_ms, gram_ms, nt_ms, os_ms = reduce_max_over_ranks(
-        [total_ms, stream_ms, gram_ms, nt_ms, os_ms], device=dev)
+    sec_ms = {k: 0.0 for k in SECTIONS}
+    for m in marks:
+        for (_, e0), (name, e1) in zip(m[:-1], m[1:]):
+            sec_ms[name] += e0.elapsed_time(e1) / args.steps
+    vals = reduce_max_over_ranks([total_ms] + [sec_ms[k] for k in SECTIONS], device=dev)
+    total_ms = vals[0]
+    sec_ms = dict(zip(SECTIONS, vals[1:]))
+    timed_s = total_ms * 1e-3
 
-    # the two tensor-core kernels one by one (outside the timed steps): the call without a
+    # the tensor-core kernels of one layer one by one (outside the timed steps): the call without a
     # sum buffer runs the Gram kernel alone, the difference to the full call is the GEMM
     reps = 20
-    g0, g1, g2 = ev(), ev(), ev()
+    g0, g1, g2, g3, g4 = ev(), ev(), ev(), ev(), ev()
+    torch.cuda.synchronize()
     g0.record(stream)
     for _ in range(reps):
         ctx.gram_sqnorm(X, D, n_layer)
@@ -305,21 +388,25 @@ def run_ours(args, rank, world, local_rank):
         ctx.gram_sqnorm(X, D, n_layer, grad_sum=S_layer, accumulate_sum=True)
     g2.record(stream)
     torch.cuda.synchronize()
-    g3 = ev()
+    g3.record(stream)
     for _ in range(reps):
         ctx.linear_sqnorm(X, D, n_layer, grad_sum=S_layer, accumulate_sum=True, method="direct")
-    g3.record(stream)
+    g4.record(stream)
     torch.cuda.synchronize()
     gram_only_ms = g0.elapsed_time(g1) / reps
     mean_grad_ms = max(g1.elapsed_time(g2) / reps - gram_only_ms, 1e-6)
-    direct_ms = g2.elapsed_time(g3) / reps
+    direct_ms = g3.elapsed_time(g4) / reps
 
-    nt_bytes, os_bytes = algorithmic_bytes()
+    ab = algorithmic_bytes()
     peaks = load_peaks()
-    value = aggregate_throughput(nt_bytes + os_bytes, world, stream_ms * 1e-3) / 1e9
+    stream_bytes = sum(ab.values())
+    stream_ms = sec_ms["nt2"] + sec_ms["os2"] + sec_ms["os5"] + sec_ms["acc5"]
+    value = aggregate_throughput(stream_bytes, world, stream_ms * 1e-3) / 1e9
     sym, executed, mg = gram_flops()
+    mflops, mlaunches = model_flops()
 
-    # ---- end to end through the host-memory entry points (rank-local pinned buffers)
+    # ---- end to end through the host-memory entry points (rank-local pinned buffers): the
+    # configs[1] pair, whose host copies (8.3 GB) fit any host; the other sections have no host form
     e2e = None
     if not args.no_e2e:
         Gh = torch.empty((NT_B, NT_P), dtype=torch.float32).pin_memory()
@@ -327,72 +414,100 @@ def run_ours(args, rank, world, local_rank):
         th_h = theta.cpu().pin_memory()
         v_h = mom.cpu().pin_memory()
         inst_h = [t.cpu().pin_memory() for t in inst]
-        reps = max(1, min(args.steps, 3))
+        ereps = max(1, min(args.steps, 3))
         ctx.norm_test_host(Gh, params[0])                   # warm-up: allocates the staging buffers
         ctx.outer_step_host(inst_h, th_h, v_h, lr=LR, momentum=MU)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        for _ in range(reps):
-            ctx.norm_test_host(Gh, params[0])
-            for p in params[1:]:
-                pass                                        # the eta sweep needs no further data movement
+        for _ in range(ereps):
+            ctx.norm_test_host(Gh, params[0])               # the eta sweep needs no further data movement
             ctx.outer_step_host(inst_h, th_h, v_h, lr=LR, momentum=MU)
         torch.cuda.synchronize()
-        e2e_s = reduce_max_over_ranks([(time.perf_counter() - t0) / reps], device=dev)[0]
-        e2e = {"value": aggregate_throughput(nt_bytes + os_bytes, world, e2e_s) / 1e9, "unit": UNIT,
-               "h2d_bytes_per_step": nt_bytes + (2 * OUT_K + 8) * OUT_P,
-               "d2h_bytes_per_step": 8 * OUT_P + 80, "ms_per_step": e2e_s * 1e3, "steps": reps}
+        e2e_s = reduce_max_over_ranks([(time.perf_counter() - t0) / ereps], device=dev)[0]
+        e2e = {"value": aggregate_throughput(ab["nt2"] + ab["os2"], world, e2e_s) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": ab["nt2"] + (2 * OUT_K + 8) * OUT_P,
+               "d2h_bytes_per_step": 8 * OUT_P + 80, "ms_per_step": e2e_s * 1e3, "steps": ereps,
+               "workload": "configs[1] pair through adloco_norm_test_host + adloco_outer_step_host (pinned host buffers)"}
         del Gh, th_h, v_h, inst_h
 
     if rank != 0:
         return
-    nt_gbs = nt_bytes / (nt_ms * 1e-3) / 1e9
-    os_gbs = os_bytes / (os_ms * 1e-3) / 1e9
+
+    # the tensor peak that fits the timed region: the sustained figure when the region lasts a second or
+    # more, or when the sampled clocks show the power cap holding the SM clock below 95 % of its maximum
+    # (the step's tensor-core sections reach the cap within tens of milliseconds); else the burst figure
+    burst, sustained = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+    capped = ("sw_power_cap" in clocks.get("reasons", []) and clocks.get("sm_mhz") and clocks.get("sm_max_mhz")
+              and clocks["sm_mhz"] < 0.95 * clocks["sm_max_mhz"])
+    regime = "sustained" if (timed_s >= 1.0 or capped) else "burst"
+    tpeak = burst if regime == "burst" else sustained
+
+    def tensor_entry(flops, ms, peak, **extra):
+        tf = flops / (ms * 1e-3) / 1e12
+        d = {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+             "frac_of_burst": tf / burst, "frac_of_sustained": tf / sustained, "algorithmic_flops": flops}
+        d.update(extra)
+        return d
+
+    def hbm_entry(nbytes, ms, **extra):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        d = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+             "frac_of_nominal_8TBs": gbs / 8000.0, "algorithmic_bytes": nbytes}
+        d.update(extra)
+        return d
+
+    model_ms = sec_ms["model4"]
+    kernels = {
+        "norm_test_kernel": hbm_entry(ab["nt2"], sec_ms["nt2"], ms_per_launch=sec_ms["nt2"], section="configs[1] norm test + eta sweep",
+                                      traffic=NT_TRAFFIC_BYTES_PER_ELEMENT * NT_B * NT_P),
+        "outer_step_kernel": hbm_entry(ab["os2"], sec_ms["os2"], ms_per_launch=sec_ms["os2"], section="configs[1] outer step K=8"),
+        "outer_step_kernel_large": hbm_entry(ab["os5"], sec_ms["os5"], ms_per_launch=sec_ms["os5"], section="configs[4] outer step K=4, P=1.3e9"),
+        "norm_test_kernel_micro": hbm_entry(ab["acc5"], sec_ms["acc5"], ms_per_launch=sec_ms["acc5"] / C5_MICRO,
+                                            section="configs[4] accumulate x8 + finalize (incl. the reset of S)"),
+        "gram_path": tensor_entry(sym + mg, sec_ms["gram3"], tpeak, ms_per_step=sec_ms["gram3"],
+                                  executed_tflops=(executed + mg) / (sec_ms["gram3"] * 1e-3) / 1e12, peak_regime=regime,
+                                  includes="configs[2]: reset + gram + mean-grad + accumulate + finalize, inside the step"),
+        "whole_model_finalize": {"ms_per_step": sec_ms["fin4"], "includes": "reset of 48 sum buffers (340 MB), 4 accumulate "
+                                 "calls, squared norm of the sums (340 MB) and the batch rule"},
+        "gram_sqnorm_kernel": tensor_entry(sym, gram_only_ms, burst, ms_per_launch=gram_only_ms,
+                                           executed_tflops=executed / (gram_only_ms * 1e-3) / 1e12,
+                                           timed="alone, 20 launches back to back (a burst), incl. the memset of n"),
+        "mean_grad_kernel": tensor_entry(mg, mean_grad_ms, burst, ms_per_launch=mean_grad_ms,
+                                         timed="alone: full call minus the Gram-only call"),
+        "direct_sqnorm_kernel_one_layer": tensor_entry(mg, direct_ms, burst, ms_per_launch=direct_ms,
+                                                       timed="alone, 20 launches back to back: adloco_linear_sqnorm(direct) on "
+                                                             "the configs[2] layer, same n_i and S as gram + mean-grad"),
+    }
+    # the dominant kernel of the step by time: the direct per-sample-gradient GEMM of the whole model
+    roofline = tensor_entry(mflops / mlaunches, model_ms / mlaunches, tpeak, kernel="direct_sqnorm_kernel",
+                            ms_per_launch=model_ms / mlaunches, launches_per_step=mlaunches, peak_regime=regime,
+                            peak_source=peaks["source"], traffic=None,
+                            section="configs[3]: 192 launches per step (48 layers x 4 micro-batches), mean over the launches; "
+                                    "flops per launch = 2 b T d_in d_out averaged over the four layer shapes")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 (streaming sections, fp64 combines); bf16 x bf16 -> f32 (tensor-core sections)",
+        "data": "synthetic",
         "config": workload_config(),
         "clocks": clocks,
         "gpu_launches": launches,
+        "timed_region_s": timed_s,
         "stream_ms_per_step": stream_ms,
-        "roofline": {"bound": "hbm", "kernel": "norm_test_kernel", "achieved": nt_gbs, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": nt_gbs / peaks["hbm_gbs"],
-                     "traffic": NT_TRAFFIC_BYTES_PER_ELEMENT * NT_B * NT_P,
-                     "peak_source": peaks["source"], "ms_per_launch": nt_ms, "algorithmic_bytes": nt_bytes},
-        "kernels": {
-            "outer_step_kernel": {"bound": "hbm", "achieved": os_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                  "frac": os_gbs / peaks["hbm_gbs"], "ms_per_launch": os_ms,
-                                  "algorithmic_bytes": os_bytes},
-            "gram_path": {"bound": "tensor", "ms_per_step": gram_ms,
-                          "achieved": (sym + mg) / (gram_ms * 1e-3) / 1e12,
-                          "executed_tflops": (executed + mg) / (gram_ms * 1e-3) / 1e12,
-                          "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                          "frac": (sym + mg) / (gram_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
-                          "algorithmic_flops": sym + mg, "includes": "gram + mean-grad + accumulate + finalize"},
-            "gram_sqnorm_kernel": {"bound": "tensor", "ms_per_launch": gram_only_ms,
-                                   "achieved": sym / (gram_only_ms * 1e-3) / 1e12,
-                                   "executed_tflops": executed / (gram_only_ms * 1e-3) / 1e12,
-                                   "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                                   "frac": sym / (gram_only_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                                   "algorithmic_flops": sym, "timed": "alone, back to back, incl. the memset of n"},
-            "mean_grad_kernel": {"bound": "tensor", "ms_per_launch": mean_grad_ms,
-                                 "achieved": mg / (mean_grad_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
-                                 "unit": "TFLOP/s", "frac": mg / (mean_grad_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                                 "algorithmic_flops": mg, "timed": "full call minus the Gram-only call"},
-            "direct_sqnorm_kernel": {"bound": "tensor", "ms_per_launch": direct_ms,
-                                     "achieved": mg / (direct_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
-                                     "unit": "TFLOP/s", "frac": mg / (direct_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                                     "algorithmic_flops": mg,
-                                     "timed": "adloco_linear_sqnorm(direct): same n_i and S as gram + mean-grad"},
-        },
-        "last_result": {"stat": last.stat, "b_req": last.b_req, "flags": last.flags},
+        "tensor_ms_per_step": sec_ms["gram3"] + sec_ms["model4"] + sec_ms["fin4"],
+        "section_ms": sec_ms,
+        "ms_x_sm_mhz": (total_ms / args.steps) * clocks["sm_mhz"] if clocks.get("sm_mhz") else None,
+        "roofline": roofline,
+        "kernels": kernels,
+        "last_result": {"stat": res5.stat, "b_req": res5.b_req, "flags": res5.flags},
     }
     if e2e is not None:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
-        gbs, ms, threads, sample = oracle_sample_run(2, 1)
-        line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+        gbs, ms, info = oracle_sample_run(2, 1)
+        line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": info["cores"], "kind": "oracle", "sample": info["sample"],
+                                "blas_pool_threads": info["blas_pool_threads"], "cores_note": info["cores_note"]}
     print(json.dumps(line), flush=True)
 
 
@@ -628,7 +743,7 @@ def run_table(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
@@ -638,8 +753,10 @@ def main():
                     help="profiling case: same kernels on inputs of a few hundred MB (not a bench value)")
     args = ap.parse_args()
     if args.small:
-        global NT_P, OUT_P
+        global NT_P, OUT_P, C4_SHAPES, C4_MICRO, C5_P, C5_MICRO, C5_ACC_P
         NT_P, OUT_P = 1 << 21, 1 << 24      # the Gram layer (252 MB) stays at its full size
+        C4_SHAPES, C4_MICRO = list(W.GPT2_SMALL_BLOCK_LINEARS), 1     # one transformer block, one micro-batch
+        C5_P, C5_MICRO, C5_ACC_P = 1 << 25, 2, 1 << 21
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -48,8 +48,11 @@ def test_single_process_is_the_identity():
     import bench
     assert bench.reduce_max_over_ranks([3.0, 1.0]) == [3.0, 1.0]
     assert bench.aggregate_throughput(4.0, 1, 2.0) == 2.0
-    nt, outer = bench.algorithmic_bytes()
-    assert nt == 4 * 64 * (1 << 24) and outer == (2 * 8 + 16) * 124_439_808
+    ab = bench.algorithmic_bytes()
+    assert ab["nt2"] == 4 * 64 * (1 << 24) and ab["os2"] == (2 * 8 + 16) * 124_439_808
+    assert ab["os5"] == (2 * 4 + 16) * 1_300_000_000 and ab["acc5"] == 8 * (4 * 32 + 8) * (1 << 22)
+    flops, launches = bench.model_flops()
+    assert launches == 192 and flops == 4 * 12 * 2 * 32 * 1024 * (768 * 2304 + 768 * 768 + 2 * 768 * 3072)
 
 
 def test_shard_bounds_partition_the_vector():
