@@ -11,9 +11,9 @@ sizes of the workload configurations:
      (X bf16 [32,1024,768], Delta bf16 [32,1024,3072]), accumulated into a
      switch-mode accumulator and finalised into one test;
   4. the whole-model test in switch mode: 12 blocks x 4 linear layers x 4
-     micro-batches of 32 sequences through adloco_linear_sqnorm (automatic
-     route), per-sample norms accumulated over layers, gradient sums over
-     micro-batches, one test at the end;
+     micro-batches of 32 sequences through adloco_linear_sqnorm_group (automatic
+     route, one launch per micro-batch), per-sample norms accumulated over
+     layers, gradient sums over micro-batches, one test at the end;
   5. outer step over K=4 bf16 instances of a 1.3B-parameter vector, in place;
   6. the norm test over 8 accumulated micro-batches of 32 x 2^22 fp32 gradients.
 The headline value is the HBM throughput of the streaming sections (1, 2, 5, 6):
@@ -80,9 +80,9 @@ def gram_flops():
 
 def model_flops():
     """Algorithmic flops of the whole-model test by the direct route: one GEMM
-    2 b T d_in d_out per (layer, micro-batch)."""
+    2 b T d_in d_out per (layer, micro-batch); one grouped launch per micro-batch."""
     per_mb = sum(2 * C4_B * GR_T * di * do for di, do in C4_SHAPES)
-    return per_mb * C4_MICRO, len(C4_SHAPES) * C4_MICRO
+    return per_mb * C4_MICRO, C4_MICRO
 
 
 def reduce_max_over_ranks(values, device="cpu"):
@@ -245,7 +245,7 @@ def workload_config():
                         "momentum, lr 0.7, Nesterov 0.9, in place) and the norm test over 8 accumulated micro-batches of "
                         "32 x 4,194,304 fp32; configs[3] whole-model switch mode: 12 blocks x 4 linear layers "
                         "(768->2304, 768->768, 768->3072, 3072->768; T=1024 bf16) x 4 micro-batches of 32 through "
-                        "adloco_linear_sqnorm(auto), accumulated and tested once; configs[1] streaming scale-up: norm test "
+                        "adloco_linear_sqnorm_group(auto), accumulated and tested once; configs[1] streaming scale-up: norm test "
                         "B=64 P=16,777,216 fp32 (eta 0.1/0.5/1.0) + outer step K=8 bf16 P=124,439,808; configs[2] Gram layer "
                         "B=32 T=1024 768->3072 bf16 (Gram identity + mean-gradient GEMM). value = bytes of the four streaming "
                         "sections / their device time; the tensor-core sections are reported in roofline and kernels",
@@ -284,6 +284,7 @@ def run_ours(args, rank, world, local_rank):
     data4 = [[W.linear_layer(C4_B, GR_T, di, do, seed=1000 * j + l + 7 * rank, device=dev)
               for l, (di, do) in enumerate(C4_SHAPES)] for j in range(C4_MICRO)]
     sums4 = [torch.zeros(do, di, device=dev) for di, do in C4_SHAPES]
+    groups4 = [ctx.make_layer_group([(Xl, Dl, S) for (Xl, Dl), S in zip(data4[j], sums4)]) for j in range(C4_MICRO)]
     acc4 = A.Accumulator(ctx, sums4)
     n_mb = torch.zeros(C4_B, device=dev)
     p4 = A.make_params(0.5, b_cur=C4_B * C4_MICRO, b_max=32)
@@ -318,13 +319,11 @@ def run_ours(args, rank, world, local_rank):
         acc.accumulate(per_sample_sqnorm=n_layer)
         acc.finalize(gparams, sync=False)
         mark("gram3")
-        # configs[3]: whole model, 4 micro-batches x 48 layers, one test
+        # configs[3]: whole model, 4 micro-batches x 48 layers (one grouped launch per micro-batch), one test
         acc4.reset()
         mark("fin4")
         for j in range(C4_MICRO):
-            for l, (Xl, Dl) in enumerate(data4[j]):
-                ctx.linear_sqnorm(Xl, Dl, n_mb, accumulate_norms=(l > 0), grad_sum=sums4[l], accumulate_sum=True,
-                                  method="auto")
+            ctx.linear_sqnorm_group(groups4[j], n_mb, method="auto", accumulate_sum=True)
             mark("model4")
             acc4.accumulate(per_sample_sqnorm=n_mb)
             if j == C4_MICRO - 1:
@@ -378,7 +377,7 @@ def run_ours(args, rank, world, local_rank):
     # the tensor-core kernels of one layer one by one (outside the timed steps): the call without a
     # sum buffer runs the Gram kernel alone, the difference to the full call is the GEMM
     reps = 20
-    g0, g1, g2, g3, g4 = ev(), ev(), ev(), ev(), ev()
+    g0, g1, g2, g3, g4, g5 = ev(), ev(), ev(), ev(), ev(), ev()
     torch.cuda.synchronize()
     g0.record(stream)
     for _ in range(reps):
@@ -392,10 +391,14 @@ def run_ours(args, rank, world, local_rank):
     for _ in range(reps):
         ctx.linear_sqnorm(X, D, n_layer, grad_sum=S_layer, accumulate_sum=True, method="direct")
     g4.record(stream)
+    for _ in range(reps):
+        ctx.linear_sqnorm(X, D, n_layer, grad_sum=S_layer, accumulate_sum=True, method="pair")
+    g5.record(stream)
     torch.cuda.synchronize()
     gram_only_ms = g0.elapsed_time(g1) / reps
     mean_grad_ms = max(g1.elapsed_time(g2) / reps - gram_only_ms, 1e-6)
     direct_ms = g3.elapsed_time(g4) / reps
+    pair_ms = g4.elapsed_time(g5) / reps
 
     ab = algorithmic_bytes()
     peaks = load_peaks()
@@ -477,13 +480,16 @@ def run_ours(args, rank, world, local_rank):
         "direct_sqnorm_kernel_one_layer": tensor_entry(mg, direct_ms, burst, ms_per_launch=direct_ms,
                                                        timed="alone, 20 launches back to back: adloco_linear_sqnorm(direct) on "
                                                              "the configs[2] layer, same n_i and S as gram + mean-grad"),
+        "direct_pair_kernel_one_layer": tensor_entry(mg, pair_ms, burst, ms_per_launch=pair_ms,
+                                                     timed="alone, 20 launches back to back: adloco_linear_sqnorm(pair) on the "
+                                                           "configs[2] layer (256 x 256 tiles over CTA pairs)"),
     }
     # the dominant kernel of the step by time: the direct per-sample-gradient GEMM of the whole model
-    roofline = tensor_entry(mflops / mlaunches, model_ms / mlaunches, tpeak, kernel="direct_sqnorm_kernel",
+    roofline = tensor_entry(mflops / mlaunches, model_ms / mlaunches, tpeak, kernel="direct_group_kernel",
                             ms_per_launch=model_ms / mlaunches, launches_per_step=mlaunches, peak_regime=regime,
                             peak_source=peaks["source"], traffic=None,
-                            section="configs[3]: 192 launches per step (48 layers x 4 micro-batches), mean over the launches; "
-                                    "flops per launch = 2 b T d_in d_out averaged over the four layer shapes")
+                            section="configs[3]: one launch per micro-batch over its 48 layers (adloco_linear_sqnorm_group, "
+                                    "automatic route); flops per launch = sum over the layers of 2 b T d_in d_out")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,

@@ -259,12 +259,40 @@ int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
  *                         W, before the mean) is formed in tensor memory, squared and
  *                         summed into n_i and added into S on chip; G_i never reaches HBM.
  *                         One GEMM of 2 B T d_in d_out flops gives both outputs.
+ *   ADLOCO_LINEAR_DIRECT_PAIR  the direct route with 256 x 256 tiles, each shared by the two
+ *                         SMs of a thread-block cluster (each loads half of the operands);
+ *                         ADLOCO_ERR_UNSUPPORTED where cluster launches are not available.
  *   ADLOCO_LINEAR_AUTO    whichever executes fewer tensor-core flops for the shape
  *                         (direct wins when T exceeds about d_in d_out / (d_in + d_out)). */
-enum { ADLOCO_LINEAR_AUTO = 0, ADLOCO_LINEAR_GRAM = 1, ADLOCO_LINEAR_DIRECT = 2 };
+enum { ADLOCO_LINEAR_AUTO = 0, ADLOCO_LINEAR_GRAM = 1, ADLOCO_LINEAR_DIRECT = 2, ADLOCO_LINEAR_DIRECT_PAIR = 3 };
 int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                          int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
                          int accumulate_sum, int method, void* stream);
+
+/* One linear layer of a group: X dev bf16 [B, T, d_in], D dev bf16 [B, T, d_out],
+ * grad_sum dev float [d_out, d_in] or NULL; d_in, d_out multiples of 8. */
+typedef struct {
+    const void* X;
+    const void* D;
+    int64_t d_in;
+    int64_t d_out;
+    float* grad_sum;
+} adloco_linear_layer;
+
+/* All linear layers of one (micro-)batch in one call (Eq. 1 applied per weight matrix; a
+ * sample's gradient is the concatenation over the layers, so its squared norm adds up):
+ *   per_sample_sqnorm[i] (+)= sum over the layers of ||D_i^T X_i||_F^2,
+ *   layers[l].grad_sum   (+)= sum_i D_i^T X_i   for every layer that gives a buffer.
+ *   layers   HOST array of n_layers entries (read during the call); all layers share B and T
+ *   method   ADLOCO_LINEAR_DIRECT, ADLOCO_LINEAR_DIRECT_PAIR or ADLOCO_LINEAR_AUTO (the pair
+ *            kernel where available, else the direct one)
+ * The direct route runs the whole group as one persistent launch per 48 layers: the work
+ * items of all layers are dealt to the SMs from one list, so small layers pay no launch of
+ * their own and layers whose tile count does not divide the SM count leave no SM idle.
+ * accumulate_norms / accumulate_sum as in adloco_gram_sqnorm, applied to every layer. */
+int adloco_linear_sqnorm_group(adloco_ctx* ctx, const adloco_linear_layer* layers, int32_t n_layers, int64_t B,
+                               int64_t T, float* per_sample_sqnorm, int accumulate_norms, int accumulate_sum,
+                               int method, void* stream);
 
 /* Per-sample gradient norms of a vector parameter of width d that acts at every
  * token (Eq. 1 applied to that parameter): a bias, g_i = sum_t delta_{i,t} (X = NULL),

@@ -23,7 +23,7 @@ FLAG_GROW, FLAG_ACCUMULATE, FLAG_UNDEFINED, FLAG_ZERO_MEAN, FLAG_NONFINITE = 1, 
 EXPORTS = (
     "adloco_create", "adloco_destroy", "adloco_status_string", "adloco_last_cuda_error", "adloco_launch_count",
     "adloco_set_wait_limit", "adloco_device_status",
-    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_inner_product_test", "adloco_gram_sqnorm", "adloco_linear_sqnorm", "adloco_vector_param_sqnorm", "adloco_embedding_sqnorm",
+    "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_inner_product_test", "adloco_gram_sqnorm", "adloco_linear_sqnorm", "adloco_linear_sqnorm_group", "adloco_vector_param_sqnorm", "adloco_embedding_sqnorm",
     "adloco_accum_create", "adloco_accum_reset", "adloco_accum_destroy", "adloco_accumulate",
     "adloco_accum_finalize", "adloco_outer_step", "adloco_outer_step_host", "adloco_check_merge", "adloco_merge",
 )
@@ -63,6 +63,14 @@ class IpResult(C.Structure):
                 ("b_ip", C.c_int64), ("b_aug", C.c_int64), ("flags", C.c_uint32), ("device_status", C.c_int32)]
 
 
+class LinearLayer(C.Structure):
+    _fields_ = [("X", C.c_void_p), ("D", C.c_void_p), ("d_in", C.c_int64), ("d_out", C.c_int64),
+                ("grad_sum", C.c_void_p)]
+
+
+LINEAR_METHODS = {"auto": 0, "gram": 1, "direct": 2, "pair": 3}
+
+
 class AdlocoError(RuntimeError):
     def __init__(self, status: int, msg: str):
         super().__init__(msg)
@@ -96,6 +104,7 @@ def load_library() -> C.CDLL:
         "adloco_inner_product_test": (C.c_int, [vp, vp, C.c_int, i64, i64, i64, C.POINTER(IpParams), vp, vp, vp, vp, vp, vp]),
         "adloco_gram_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
         "adloco_linear_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, C.c_int, vp]),
+        "adloco_linear_sqnorm_group": (C.c_int, [vp, C.POINTER(LinearLayer), i32, i64, i64, vp, C.c_int, C.c_int, C.c_int, vp]),
         "adloco_vector_param_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
         "adloco_embedding_sqnorm": (C.c_int, [vp, vp, vp, i64, i64, i64, i64, vp, C.c_int, vp, C.c_int, vp]),
         "adloco_accum_create": (C.c_int, [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), i32]),
@@ -257,16 +266,41 @@ class Context:
 
     def linear_sqnorm(self, X, D, per_sample_sqnorm, *, method="auto", accumulate_norms=False, grad_sum=None,
                       accumulate_sum=False, stream=None):
-        """adloco_linear_sqnorm: method is "auto", "gram" or "direct"."""
+        """adloco_linear_sqnorm: method is "auto", "gram", "direct" or "pair"."""
         B, T, d_in = X.shape
         d_out = D.shape[2]
         if X.dtype != torch.bfloat16 or D.dtype != torch.bfloat16 or not X.is_contiguous() or not D.is_contiguous():
             raise AdlocoError(ERR_INVALID_ARG, "X and D must be contiguous bfloat16")
-        code = {"auto": 0, "gram": 1, "direct": 2}[method]
+        code = LINEAR_METHODS[method]
         rc = self.lib.adloco_linear_sqnorm(self.h, _ptr(X), _ptr(D), B, T, d_in, d_out, _ptr(per_sample_sqnorm),
                                            int(accumulate_norms), _ptr(grad_sum), int(accumulate_sum), code,
                                            _stream(stream))
         self.check(rc, "adloco_linear_sqnorm")
+
+    def make_layer_group(self, layers):
+        """Marshals [(X, D, grad_sum or None), ...] (bf16 [B, T, d] tensors of one B and T) into the
+        array adloco_linear_sqnorm_group takes; the result can be reused while the tensors live."""
+        arr = (LinearLayer * len(layers))()
+        B, T = layers[0][0].shape[0], layers[0][0].shape[1]
+        for k, (X, D, S) in enumerate(layers):
+            if (X.dtype != torch.bfloat16 or D.dtype != torch.bfloat16 or not X.is_contiguous() or not D.is_contiguous()
+                    or X.shape[:2] != (B, T) or D.shape[:2] != (B, T)):
+                raise AdlocoError(ERR_INVALID_ARG, "X and D must be contiguous bfloat16 [B, T, d] with one B and T")
+            if S is not None and (S.dtype != torch.float32 or tuple(S.shape) != (D.shape[2], X.shape[2]) or not S.is_contiguous()):
+                raise AdlocoError(ERR_INVALID_ARG, "grad_sum must be contiguous float32 [d_out, d_in]")
+            arr[k] = LinearLayer(X.data_ptr(), D.data_ptr(), X.shape[2], D.shape[2], None if S is None else S.data_ptr())
+        return arr, len(layers), B, T
+
+    def linear_sqnorm_group(self, group, per_sample_sqnorm, *, method="auto", accumulate_norms=False,
+                            accumulate_sum=False, stream=None):
+        """adloco_linear_sqnorm_group on a group from make_layer_group (or a list of (X, D, S) triples);
+        method is "auto", "direct" or "pair"."""
+        if isinstance(group, (list, tuple)) and not isinstance(group[0], C.Array):
+            group = self.make_layer_group(group)
+        arr, n, B, T = group
+        rc = self.lib.adloco_linear_sqnorm_group(self.h, arr, n, B, T, _ptr(per_sample_sqnorm), int(accumulate_norms),
+                                                 int(accumulate_sum), LINEAR_METHODS[method], _stream(stream))
+        self.check(rc, "adloco_linear_sqnorm_group")
 
     def vector_param_sqnorm(self, D, per_sample_sqnorm, *, X=None, accumulate_norms=False, grad_sum=None,
                             accumulate_sum=False, stream=None):

@@ -44,6 +44,15 @@ int ensure_staging(adloco_ctx* ctx, size_t bytes_each) {
 
 constexpr size_t kPanelBytes = 64u << 20;  // staging panel of the host-memory entry points
 
+// thread-block clusters of two CTAs need compute capability 9.0 or later and the launch attribute
+bool pair_launch_ok(adloco_ctx* ctx) {
+    if (ctx->pair_ok < 0) {
+        int v = 0;
+        ctx->pair_ok = (cudaDeviceGetAttribute(&v, cudaDevAttrClusterLaunch, ctx->device) == cudaSuccess && v != 0) ? 1 : 0;
+    }
+    return ctx->pair_ok == 1;
+}
+
 }  // namespace
 
 extern "C" {
@@ -84,6 +93,7 @@ int adloco_create(adloco_ctx** out, int device) {
     ok = ok && cudaMalloc(&ctx->scratch_sums, sizeof(adloco_test_sums)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->gemm_status, 64) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->n_scratch, kMaxBatchRows * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->sched_counters, kSchedCounters * sizeof(int)) == cudaSuccess;
     ok = ok && cudaMemset(ctx->ticket, 0, 64) == cudaSuccess;
     ok = ok && cudaMemset(ctx->gemm_status, 0, 64) == cudaSuccess;
     ok = ok && cudaMemset(ctx->scratch_sums, 0, sizeof(adloco_test_sums)) == cudaSuccess;
@@ -102,6 +112,8 @@ int adloco_destroy(adloco_ctx* ctx) {
     cudaFree(ctx->scratch_sums);
     cudaFree(ctx->gemm_status);
     cudaFree(ctx->n_scratch);
+    cudaFree(ctx->sched_counters);
+    free_tensor_map_cache(ctx);
     HostStaging& s = ctx->staging;
     for (int i = 0; i < 2; ++i) {
         cudaFree(s.dev[i]);
@@ -312,7 +324,8 @@ int adloco_embedding_sqnorm(adloco_ctx* ctx, const int32_t* token_ids, const voi
 int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                          int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
                          int accumulate_sum, int method, void* stream) {
-    if (method != ADLOCO_LINEAR_AUTO && method != ADLOCO_LINEAR_GRAM && method != ADLOCO_LINEAR_DIRECT)
+    if (method != ADLOCO_LINEAR_AUTO && method != ADLOCO_LINEAR_GRAM && method != ADLOCO_LINEAR_DIRECT &&
+        method != ADLOCO_LINEAR_DIRECT_PAIR)
         return ADLOCO_ERR_INVALID_ARG;
     if (!ctx || !X || !D || !per_sample_sqnorm) return ADLOCO_ERR_INVALID_ARG;
     if (B < 1 || T < 1 || d_in < 1 || d_out < 1) return ADLOCO_ERR_INVALID_ARG;
@@ -340,8 +353,34 @@ int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
     if (!aligned16(X) || !aligned16(D)) return ADLOCO_ERR_ALIGNMENT;
     if (grad_sum && !aligned16(grad_sum)) return ADLOCO_ERR_ALIGNMENT;
     DeviceGuard g(ctx->device);
+    if (method == ADLOCO_LINEAR_DIRECT_PAIR && !pair_launch_ok(ctx)) return ADLOCO_ERR_UNSUPPORTED;
     return launch_direct_sqnorm(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, grad_sum,
-                                accumulate_sum, static_cast<cudaStream_t>(stream));
+                                accumulate_sum, method == ADLOCO_LINEAR_DIRECT_PAIR, static_cast<cudaStream_t>(stream));
+}
+
+int adloco_linear_sqnorm_group(adloco_ctx* ctx, const adloco_linear_layer* layers, int32_t n_layers, int64_t B,
+                               int64_t T, float* per_sample_sqnorm, int accumulate_norms, int accumulate_sum,
+                               int method, void* stream) {
+    if (method != ADLOCO_LINEAR_AUTO && method != ADLOCO_LINEAR_DIRECT && method != ADLOCO_LINEAR_DIRECT_PAIR)
+        return ADLOCO_ERR_INVALID_ARG;
+    if (!ctx || !layers || n_layers < 1 || !per_sample_sqnorm || B < 1 || T < 1) return ADLOCO_ERR_INVALID_ARG;
+    if (B > (1 << 30) || T > (1 << 30) || n_layers > (1 << 20)) return ADLOCO_ERR_UNSUPPORTED;
+    for (int l = 0; l < n_layers; ++l) {
+        const adloco_linear_layer& L = layers[l];
+        if (!L.X || !L.D || L.d_in < 1 || L.d_out < 1) return ADLOCO_ERR_INVALID_ARG;
+        if ((L.d_in % 8) != 0 || (L.d_out % 8) != 0 || L.d_in > (1 << 30) || L.d_out > (1 << 30)) return ADLOCO_ERR_UNSUPPORTED;
+        if (!aligned16(L.X) || !aligned16(L.D) || (L.grad_sum && !aligned16(L.grad_sum))) return ADLOCO_ERR_ALIGNMENT;
+    }
+    DeviceGuard g(ctx->device);
+    int pair = 0;
+    if (method == ADLOCO_LINEAR_DIRECT_PAIR) {
+        if (!pair_launch_ok(ctx)) return ADLOCO_ERR_UNSUPPORTED;
+        pair = 1;
+    } else if (method == ADLOCO_LINEAR_AUTO) {
+        pair = pair_launch_ok(ctx) ? 1 : 0;
+    }
+    return launch_direct_group(ctx, layers, n_layers, B, T, per_sample_sqnorm, accumulate_norms, accumulate_sum, pair,
+                               static_cast<cudaStream_t>(stream));
 }
 
 // ---------------------------------------------------------------------------------

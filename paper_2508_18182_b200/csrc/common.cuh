@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <atomic>
 #include <stdint.h>
 #include <stdio.h>
 #include <string.h>
@@ -16,6 +17,7 @@
 namespace adloco {
 
 constexpr int kMaxInstances = 64;     // K of the outer step / merge (pointers travel as kernel arguments)
+constexpr int kSchedCounters = 1024;   // launches of the grouped kernel that may be in flight at once
 constexpr int64_t kMaxBatchRows = 4096;  // B of one materialised (micro-)batch (per-warp rows live in shared memory)
 
 // Staging buffers for the host-memory entry points (allocated on first use).
@@ -46,6 +48,10 @@ struct adloco_ctx {
     int* gemm_status = nullptr;                // device status word of the tensor-core kernels
     uint64_t wait_limit_ns = 2000000000ull;    // bound of every in-kernel wait: 2 s, far beyond any legitimate wait
     float* n_scratch = nullptr;                // [kMaxBatchRows] per-sample norms when the caller wants none
+    void* tensor_maps = nullptr;               // cache of encoded tensor maps (gram_kernels.cu owns the type)
+    int pair_ok = -1;                          // CTA-pair launches possible on this device: -1 not asked yet
+    int* sched_counters = nullptr;             // [kSchedCounters] work counters of the grouped tensor-core kernel
+    std::atomic<unsigned> sched_next{0};       // next counter to hand to a launch
 
     adloco::HostStaging staging;
 };
@@ -159,7 +165,10 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
 int launch_embedding(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, int64_t T, int64_t d, int64_t V,
                      float* n, int accumulate_norms, float* S, int accumulate_sum, cudaStream_t st);
 int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
-                         int64_t d_out, float* n, int accumulate_norms, float* S, int accumulate_sum,
+                         int64_t d_out, float* n, int accumulate_norms, float* S, int accumulate_sum, int pair,
                          cudaStream_t st);
+int launch_direct_group(adloco_ctx* ctx, const adloco_linear_layer* layers, int n_layers, int64_t B, int64_t T,
+                        float* n, int accumulate_norms, int accumulate_sum, int pair, cudaStream_t st);
+void free_tensor_map_cache(adloco_ctx* ctx);
 
 }  // namespace adloco

@@ -14,6 +14,9 @@
 // Every wait is bounded; a wait that runs out raises a status word and all
 // roles leave through the common teardown.
 #include <atomic>
+#include <mutex>
+#include <new>
+#include <unordered_map>
 
 #include "common.cuh"
 #include "ptx.cuh"
@@ -22,6 +25,7 @@ namespace adloco {
 
 using namespace ptx;
 
+constexpr int kDirectGroupCap = 48;                 // layers per launch of the grouped direct kernel
 constexpr uint64_t kDrainLimitNs = 50000000ull;    // 50 ms per barrier while leaving after a time-out
 
 struct PipeState {
@@ -683,173 +687,322 @@ mean_grad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 // =====================================================================================
 // direct kernel: per-sample weight-gradient tiles formed in TMEM, never written out
 // =====================================================================================
-// For one (128 x 256 output tile, sample i) unit the contraction over the sample's
-// T tokens leaves the tile of G_i = D_i^T X_i in TMEM.  The epilogue squares and
-// sums it into n_i and adds it to a register copy of the tile of S = sum_i G_i,
-// which is flushed to global memory when the CTA moves to another tile.  One GEMM
-// (2 B T d_in d_out flops) thus yields both the per-sample norms and the gradient
-// sum; it beats the Gram route whenever T exceeds d_in d_out / (d_in + d_out).
-constexpr int DR_BM = 128;                          // d_out rows per tile
+// For one (output tile, sample i) unit the contraction over the sample's T tokens
+// leaves the tile of G_i = D_i^T X_i in TMEM.  The epilogue squares and sums it into
+// n_i and adds it to a register copy of the tile of S = sum_i G_i, which is flushed to
+// global memory when the work item ends.  One GEMM (2 B T d_in d_out flops) thus
+// yields both the per-sample norms and the gradient sum; it beats the Gram route
+// whenever T exceeds d_in d_out / (d_in + d_out).
+//
+// The kernel takes a GROUP of layers (all with the same B and T): its work list runs
+// over every layer's (chunk of samples, tile) items, so a whole micro-batch of a model is
+// one persistent launch with one ramp and one tail, and the (tile, sample) units of
+// layers whose tile count does not divide the SM count still spread evenly.  Items are
+// handed out in list order through a global counter: a worker that finishes takes the
+// next item, so all workers stay within a window of consecutive items -- the same few
+// samples of the same layer, whose operands then stay in L2 (a fixed deal lets the workers
+// drift apart over a long list and the DRAM traffic multiply).  The TMA thread draws the
+// item and passes it to the other roles through a small queue in shared memory.
+//
+// PAIR = false: one CTA per SM, tile 128 (d_out) x 256 (d_in), stage = 48 KB.
+// PAIR = true:  the two CTAs of a cluster share one MMA of 256 x 256: CTA r holds rows
+//   128 r .. 128 r + 127 of the tile in its tensor memory, loads its own 128 rows of the
+//   Delta operand and one half (128 columns) of the X operand -- 32 KB per stage for the
+//   same math, i.e. 131 flops per byte brought into shared memory instead of 87.  The even
+//   CTA issues the MMAs; byte counts of both CTAs' loads complete on its barriers; its
+//   commits release the stages and publish the accumulators in both CTAs.
+constexpr int DR_BM = 128;                          // d_out rows per CTA
 constexpr int DR_BN = 256;                          // d_in columns per tile
 constexpr int DR_BK = 64;                           // tokens per stage
-constexpr int DR_STAGES = 4;
-constexpr int DR_BOX_BYTES = 64 * DR_BK * 2;        // 8 KB
+constexpr int DR_BOX_BYTES = 64 * DR_BK * 2;        // 8 KB: 64 features x 64 tokens
 constexpr int DR_A_BYTES = (DR_BM / 64) * DR_BOX_BYTES;
-constexpr int DR_B_BYTES = (DR_BN / 64) * DR_BOX_BYTES;
-constexpr int DR_STAGE_BYTES = DR_A_BYTES + DR_B_BYTES;   // 48 KB
 constexpr int DR_BOX_OUT = 32 * 16 * 4;             // per-epilogue-warp staging box: 32 rows x 16 fp32 columns
-constexpr int DR_STAGING = 12 * DR_BOX_OUT;
-constexpr int DR_SMEM = DR_STAGES * DR_STAGE_BYTES + DR_STAGING + 1024 + 256;
-// Epilogue: three warps per TMEM lane quarter; the 16 column chunks (of 16) of a tile
-// row are split 6 / 5 / 5 among them, so a thread keeps at most 96 columns of the S
-// tile in registers (16 warps' worth of register file at 128 registers per thread).
-constexpr int DR_EPI_WARPS = 12;
-constexpr int DR_CHUNKS_MAX = 6;
+// Epilogue: four warps per TMEM lane quarter, each with four of the 16 column chunks (of
+// 16) of a tile row, so a thread keeps 64 columns of the S tile in registers.
+constexpr int DR_EPI_WARPS = 16;
+constexpr int DR_STAGING = DR_EPI_WARPS * DR_BOX_OUT;
+constexpr int DR_CHUNKS_MAX = 4;
 constexpr int DR_COLS = DR_CHUNKS_MAX * 16;
 constexpr int DR_THREADS = 64 + 32 * DR_EPI_WARPS;  // warp 0 TMA, warp 1 MMA, the rest epilogue
+constexpr uint64_t kPairGraceNs = 1000000ull;       // 1 ms: leaving after a time-out, copies in flight land long before
+constexpr int DR_SCHED_Q = 8;                       // slots of the item queue between the TMA thread and the other roles
 
-struct DirectArgs {
-    int B, T, d_in, d_out;
-    int ntm, ntn;
-    int splits, chunk, items;   // see SplitPlan
-    float* n;           // [B], +=
-    float* S;           // [d_out, d_in], += ; may be null
-    int* status;
-    uint64_t wait_ns;   // bound of every in-kernel wait
+template <bool PAIR>
+struct DirectCfg {
+    static constexpr int B_BYTES = (PAIR ? 128 : DR_BN) / 64 * DR_BOX_BYTES;   // this CTA's share of the X operand
+    static constexpr int STAGE_BYTES = DR_A_BYTES + B_BYTES;                   // 32 KB / 48 KB
+    static constexpr int STAGES = PAIR ? 6 : 4;
+    static constexpr int SMEM = STAGES * STAGE_BYTES + DR_STAGING + 1024 /*align*/ + 512 /*barriers*/;
+    static constexpr int TILE_M = PAIR ? 256 : 128;                            // d_out rows per tile
 };
 
+struct alignas(64) DirectLayerMaps {
+    CUtensorMap tmX, tmD, tmS;
+};
+struct DirectLayerMeta {
+    float* S;            // [d_out, d_in], += ; may be null
+    int d_in, d_out;
+    int ntn, tiles;      // tiles along d_in, tiles of the layer
+    int item_begin;      // first work item of the layer
+    int pad;
+};
+
+// Work item j of a layer = (chunk of samples j / tiles, tile j % tiles): all tiles of one
+// chunk of samples come first, so CTAs that run side by side read the same few samples
+// and those samples' operands stay in L2.
+template <int CAP>
+struct DirectGroupArgs {
+    DirectLayerMaps maps[CAP];
+    DirectLayerMeta meta[CAP];
+    int n_layers, B, T, kt;
+    int chunk;           // samples per work item
+    int total_items;
+    int* counter;        // zero at launch: items beyond each worker's first are drawn from it
+    float* n;            // [B], +=
+    int* status;
+    uint64_t wait_ns;    // bound of every in-kernel wait
+};
+
+struct DirectItem {
+    int layer, tm, tn, b0, b1;
+};
+
+template <int CAP>
+__device__ __forceinline__ DirectItem direct_decode(const DirectGroupArgs<CAP>& a, int item, int& layer_hint) {
+    int l = layer_hint;
+    while (l + 1 < a.n_layers && item >= a.meta[l + 1].item_begin) ++l;
+    layer_hint = l;
+    const DirectLayerMeta& m = a.meta[l];
+    const int local = item - m.item_begin;
+    const int k = local / m.tiles, tile = local - k * m.tiles;
+    DirectItem it;
+    it.layer = l;
+    it.tm = tile / m.ntn;
+    it.tn = tile - it.tm * m.ntn;
+    it.b0 = k * a.chunk;
+    it.b1 = it.b0 + a.chunk < a.B ? it.b0 + a.chunk : a.B;
+    return it;
+}
+
+template <int CAP, bool PAIR>
 __global__ void __launch_bounds__(DR_THREADS, 1)
-direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
-                     const __grid_constant__ CUtensorMap tmS, const DirectArgs a) {
+direct_group_kernel(const __grid_constant__ DirectGroupArgs<CAP> a) {
+    using Cfg = DirectCfg<PAIR>;
+    constexpr int STAGES = Cfg::STAGES;
+    constexpr int STAGE_BYTES = Cfg::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t staging_base = smem_base + DR_STAGES * DR_STAGE_BYTES;
+    const uint32_t staging_base = smem_base + STAGES * STAGE_BYTES;
     const uint32_t bar_base = staging_base + DR_STAGING;
     auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
-    auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (DR_STAGES + s); };
-    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * DR_STAGES + b); };
-    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * DR_STAGES + 2 + b); };
-    const uint32_t drain_bar = bar_base + 8u * (2 * DR_STAGES + 4);
+    auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * STAGES + 4);
+    auto sched_full = [&](uint32_t s) { return bar_base + 8u * (2 * STAGES + 5 + s); };
+    auto sched_empty = [&](uint32_t s) { return bar_base + 8u * (2 * STAGES + 5 + DR_SCHED_Q + s); };
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int sched_item[DR_SCHED_Q];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = PAIR ? cluster_cta_rank() : 0u;          // 0 = the CTA that issues the MMAs and draws the items
+    const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (uint32_t s = 0; s < DR_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), DR_EPI_WARPS); }
+        for (uint32_t s = 0; s < (uint32_t)STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (uint32_t b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), DR_EPI_WARPS * (PAIR ? 2 : 1));    // the epilogue warps of both CTAs
+        }
         mbar_init(drain_bar, 1);
+        for (uint32_t s = 0; s < (uint32_t)DR_SCHED_Q; ++s) {
+            mbar_init(sched_full(s), 1);
+            // readers of a slot: the MMA thread and the epilogue warps; over a pair also the odd
+            // CTA's TMA thread and epilogue warps
+            mbar_init(sched_empty(s), (1 + DR_EPI_WARPS) * (PAIR ? 2 : 1));
+        }
         fence_barrier_init();
-        prefetch_tmap(&tmX);
-        prefetch_tmap(&tmD);
-        if (a.S != nullptr) prefetch_tmap(&tmS);
     }
-    if (warp == 1) {
-        tmem_alloc(smem_u32(&tmem_base_slot), 512);   // two 128x256 fp32 accumulators
-        tmem_relinquish();
+    if (warp == 1) {   // two 128 x 256 fp32 accumulators
+        if constexpr (PAIR) { tmem_alloc_pair(smem_u32(&tmem_base_slot), 512); tmem_relinquish_pair(); }
+        else { tmem_alloc(smem_u32(&tmem_base_slot), 512); tmem_relinquish(); }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();    // the peer's barriers exist before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
+    const int kt = a.kt;
+    const uint32_t sched_empty_remote0 = PAIR ? map_to_cta(sched_empty(0), 0) : 0u;
 
-    const int kt = (a.T + DR_BK - 1) / DR_BK;
+    // item number k of this worker, as published by the drawing thread; -1 when the wait ran out.
+    // Called by one thread (TMA / MMA role) or by all lanes of an epilogue warp.
+    auto take_item = [&](int k, bool whole_warp) -> int {
+        const uint32_t slot = (uint32_t)k % DR_SCHED_Q, ph = ((uint32_t)k / DR_SCHED_Q) & 1u;
+        bool got = mbar_wait<PAIR>(sched_full(slot), ph, abortp, a.wait_ns);
+        if (whole_warp) got = __all_sync(0xffffffffu, got);
+        if (!got) return -1;
+        const int item = *reinterpret_cast<volatile int*>(&sched_item[slot]);
+        if (whole_warp) __syncwarp();
+        if (!whole_warp || lane == 0) {
+            if (PAIR && rank != 0) mbar_arrive_cluster(sched_empty_remote0 + 8u * slot);
+            else mbar_arrive(sched_empty(slot));
+        }
+        return item;
+    };
 
     if (warp == 0) {
         if (lane == 0) {
             PipeState ps;
             uint32_t issued = 0;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < a.items; item += gridDim.x) {
-            int64_t u0, u1;
-            item_range(item, a.splits, a.chunk, a.B, u0, u1);
-            for (int64_t u = u0; ok && u < u1; ++u) {
-                const int tile = (int)(u / a.B), i = (int)(u % a.B);
-                const int tm = tile / a.ntn, tn = tile % a.ntn;
-                for (int c = 0; c < kt; ++c) {
-                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
-                    const uint32_t sA = smem_base + ps.stage * DR_STAGE_BYTES;
-                    const uint32_t sB = sA + DR_A_BYTES;
-                    mbar_arrive_expect_tx(full_bar(ps.stage), DR_STAGE_BYTES);
-#pragma unroll
-                    for (int mb = 0; mb < DR_BM / 64; ++mb)
-                        tma_load_3d(sA + mb * DR_BOX_BYTES, &tmD, full_bar(ps.stage), tm * DR_BM + mb * 64, c * DR_BK, i);
-#pragma unroll
-                    for (int nb = 0; nb < DR_BN / 64; ++nb)
-                        tma_load_3d(sB + nb * DR_BOX_BYTES, &tmX, full_bar(ps.stage), tn * DR_BN + nb * 64, c * DR_BK, i);
-                    ++issued;
-                    ps.advance(DR_STAGES);
+            int hint = 0;
+            int item = worker;                      // the first item needs no draw
+            for (int k = 0; ok; ++k) {
+                if (rank == 0) {
+                    // publish item k to the other roles (and to the peer CTA)
+                    const uint32_t slot = (uint32_t)k % DR_SCHED_Q, ph = ((uint32_t)k / DR_SCHED_Q) & 1u;
+                    if (!mbar_wait<PAIR>(sched_empty(slot), ph ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
+                    *reinterpret_cast<volatile int*>(&sched_item[slot]) = item;
+                    if constexpr (PAIR) st_cluster_u32(map_to_cta(smem_u32(&sched_item[slot]), 1u), (uint32_t)item);
+                    mbar_arrive(sched_full(slot));
+                    if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(sched_full(slot), 1u));
+                } else {
+                    item = take_item(k, false);
+                    if (item < 0) { ok = false; break; }
                 }
-            }
+                if (item >= a.total_items) break;   // the list is exhausted: every role has been told
+                // draw the next item now, its latency hides behind this item's copies
+                int next_item = 0;
+                if (rank == 0) next_item = n_workers + atomicAdd(a.counter, 1);
+                const DirectItem it = direct_decode(a, item, hint);
+                const CUtensorMap* tmD = &a.maps[it.layer].tmD;
+                const CUtensorMap* tmX = &a.maps[it.layer].tmX;
+                const int row0 = it.tm * Cfg::TILE_M + (int)rank * DR_BM;              // this CTA's d_out rows
+                const int col0 = it.tn * DR_BN + (PAIR ? (int)rank * 128 : 0);         // this CTA's d_in columns
+                for (int i = it.b0; ok && i < it.b1; ++i) {
+                    for (int c = 0; c < kt; ++c) {
+                        if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
+                        const uint32_t sA = smem_base + ps.stage * STAGE_BYTES;
+                        const uint32_t sB = sA + DR_A_BYTES;
+                        if constexpr (PAIR) {
+                            const uint32_t bar = map_to_cta(full_bar(ps.stage), 0);
+                            if (rank == 0) mbar_arrive_expect_tx(full_bar(ps.stage), 2 * STAGE_BYTES);
+#pragma unroll
+                            for (int mb = 0; mb < DR_BM / 64; ++mb)
+                                tma_load_3d_pair(sA + mb * DR_BOX_BYTES, tmD, bar, row0 + mb * 64, c * DR_BK, i);
+#pragma unroll
+                            for (int nb = 0; nb < 2; ++nb)
+                                tma_load_3d_pair(sB + nb * DR_BOX_BYTES, tmX, bar, col0 + nb * 64, c * DR_BK, i);
+                        } else {
+                            mbar_arrive_expect_tx(full_bar(ps.stage), STAGE_BYTES);
+#pragma unroll
+                            for (int mb = 0; mb < DR_BM / 64; ++mb)
+                                tma_load_3d(sA + mb * DR_BOX_BYTES, tmD, full_bar(ps.stage), row0 + mb * 64, c * DR_BK, i);
+#pragma unroll
+                            for (int nb = 0; nb < DR_BN / 64; ++nb)
+                                tma_load_3d(sB + nb * DR_BOX_BYTES, tmX, full_bar(ps.stage), col0 + nb * 64, c * DR_BK, i);
+                        }
+                        ++issued;
+                        ps.advance(STAGES);
+                    }
+                }
+                item = next_item;
             }
             if (!ok) {
-                PipeState q = ps;
-                const uint32_t back = issued < DR_STAGES ? issued : DR_STAGES;
-                for (uint32_t r = 0; r < back; ++r) {
-                    if (q.stage == 0) { q.stage = DR_STAGES - 1; q.phase ^= 1u; } else { --q.stage; }
-                    int never = 0;
-                    mbar_wait(full_bar(q.stage), q.phase, &never, kDrainLimitNs);
+                // leaving after a time-out: let the copies still in flight land first
+                if constexpr (PAIR) {
+                    // their byte counts complete on the even CTA's barriers, which the odd CTA cannot
+                    // wait on: both sit out a grace period far beyond the flight time of a copy
+                    st_cluster_u32(map_to_cta(smem_u32(&abort_flag), rank ^ 1u), 1u);
+                    const uint64_t t0 = globaltimer_ns();
+                    while (globaltimer_ns() - t0 < kPairGraceNs) { }
+                } else {
+                    PipeState q = ps;
+                    const uint32_t back = issued < (uint32_t)STAGES ? issued : (uint32_t)STAGES;
+                    for (uint32_t r = 0; r < back; ++r) {
+                        if (q.stage == 0) { q.stage = STAGES - 1; q.phase ^= 1u; } else { --q.stage; }
+                        int never = 0;
+                        mbar_wait(full_bar(q.stage), q.phase, &never, kDrainLimitNs);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16_f32(DR_BM, DR_BN, 1, 1);   // both operands MN-major
+        if (lane == 0 && rank == 0) {
+            // both operands MN-major; over a pair the MMA spans 256 rows (128 per CTA)
+            constexpr uint32_t idesc = idesc_bf16_f32(PAIR ? 256 : DR_BM, DR_BN, 1, 1);
             PipeState ps;
             bool ok = true;
             int n_unit = 0;
-            for (int item = blockIdx.x; ok && item < a.items; item += gridDim.x) {
-            int64_t u0, u1;
-            item_range(item, a.splits, a.chunk, a.B, u0, u1);
-            for (int64_t u = u0; ok && u < u1; ++u, ++n_unit) {
-                const uint32_t buf = n_unit & 1, use = n_unit >> 1;
-                if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t acc = tmem_base + buf * 256u;
-                for (int c = 0; c < kt; ++c) {
-                    if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, a.wait_ns)) { ok = false; break; }
+            int hint = 0;
+            for (int k = 0; ok; ++k) {
+                const int item = take_item(k, false);
+                if (item < 0) { ok = false; break; }
+                if (item >= a.total_items) break;
+                const DirectItem it = direct_decode(a, item, hint);
+                for (int i = it.b0; ok && i < it.b1; ++i, ++n_unit) {
+                    const uint32_t buf = n_unit & 1, use = n_unit >> 1;
+                    if (!mbar_wait<PAIR>(tempty_bar(buf), (use & 1u) ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sA = smem_base + ps.stage * DR_STAGE_BYTES;
-                    const uint32_t sB = sA + DR_A_BYTES;
+                    const uint32_t acc = tmem_base + buf * 256u;
+                    for (int c = 0; c < kt; ++c) {
+                        if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, a.wait_ns)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t sA = smem_base + ps.stage * STAGE_BYTES;
+                        const uint32_t sB = sA + DR_A_BYTES;
 #pragma unroll
-                    for (int kk = 0; kk < DR_BK / 16; ++kk) {
-                        const uint64_t da = smem_desc_sw128(sA + kk * 2048, DR_BOX_BYTES, 1024);
-                        const uint64_t db = smem_desc_sw128(sB + kk * 2048, DR_BOX_BYTES, 1024);
-                        mma_bf16(acc, da, db, idesc, (c == 0 && kk == 0) ? 0u : 1u);
+                        for (int kk = 0; kk < DR_BK / 16; ++kk) {
+                            // MN-major, 128-byte swizzle: a token is a 128-byte row of 64 features, 8-token
+                            // groups 1024 B apart (stride offset), the next 64 features one box further
+                            // (leading offset); 16 tokens = 2 KB per MMA
+                            const uint64_t da = smem_desc_sw128(sA + kk * 2048, DR_BOX_BYTES, 1024);
+                            const uint64_t db = smem_desc_sw128(sB + kk * 2048, DR_BOX_BYTES, 1024);
+                            if constexpr (PAIR) mma_bf16_pair(acc, da, db, idesc, (c == 0 && kk == 0) ? 0u : 1u);
+                            else mma_bf16(acc, da, db, idesc, (c == 0 && kk == 0) ? 0u : 1u);
+                        }
+                        if constexpr (PAIR) mma_commit_pair(empty_bar(ps.stage), 3);   // the stage is free in both CTAs
+                        else mma_commit(empty_bar(ps.stage));
+                        ps.advance(STAGES);
                     }
-                    mma_commit(empty_bar(ps.stage));
-                    ps.advance(DR_STAGES);
+                    if (ok) {
+                        if constexpr (PAIR) mma_commit_pair(tfull_bar(buf), 3);
+                        else mma_commit(tfull_bar(buf));
+                    }
                 }
-                if (ok) mma_commit(tfull_bar(buf));
-            }
             }
             if (!ok) {
-                mma_commit(drain_bar);
+                if constexpr (PAIR) {
+                    st_cluster_u32(map_to_cta(smem_u32(&abort_flag), 1u), 1u);
+                    mma_commit_pair(drain_bar, 1);
+                } else {
+                    mma_commit(drain_bar);
+                }
                 int never = 0;
                 mbar_wait(drain_bar, 0, &never, kDrainLimitNs);
             }
         }
     } else {
-        const uint32_t q = warp & 3;            // TMEM lane quarter: rows 32q .. 32q+31 of the tile
+        const uint32_t q = warp & 3;            // TMEM lane quarter: rows 32q .. 32q+31 of this CTA's part of the tile
         const uint32_t part = (warp - 2) >> 2;  // which column slice of the tile: chunks [c_begin, c_begin + n_chunks)
-        const int c_begin = part == 0 ? 0 : (part == 1 ? 6 : 11);
-        const int n_chunks = part == 0 ? 6 : 5;
+        const int c_begin = (int)part * DR_CHUNKS_MAX;
+        constexpr int n_chunks = DR_CHUNKS_MAX;
+        const uint32_t tempty_remote0 = PAIR ? map_to_cta(tempty_bar(0), 0) : 0u;
         float sacc[DR_COLS];                    // this thread's row of the S tile (its column slice)
 #pragma unroll
         for (int e = 0; e < DR_COLS; ++e) sacc[e] = 0.f;
         int n_unit = 0;
         bool ok = true;
-        for (int item = blockIdx.x; ok && item < a.items; item += gridDim.x) {
-        int64_t u0, u1;
-        item_range(item, a.splits, a.chunk, a.B, u0, u1);
-        int64_t u = u0;
-        while (ok && u < u1) {
-            // one segment: this work item's samples of its output tile
-            const int tile = (int)(u / a.B);
-            const int64_t u_end = u1;
-            for (; u < u_end; ++u, ++n_unit) {
-                const int i = (int)(u - (int64_t)tile * a.B);
+        int hint = 0;
+        for (int k = 0; ok; ++k) {
+            const int item = take_item(k, true);
+            if (item < 0) { ok = false; break; }
+            if (item >= a.total_items) break;
+            const DirectItem it = direct_decode(a, item, hint);
+            for (int i = it.b0; i < it.b1; ++i, ++n_unit) {
                 const uint32_t buf = n_unit & 1, use = n_unit >> 1;
                 if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abortp, a.wait_ns))) { ok = false; break; }
                 tc_fence_after();
@@ -871,22 +1024,25 @@ direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar(buf));
+                if (lane == 0) {
+                    if constexpr (PAIR) mbar_arrive_cluster(tempty_remote0 + 8u * buf);   // the even CTA's barrier
+                    else mbar_arrive(tempty_bar(buf));
+                }
                 const float w = warp_sum_f(sq);
                 if (lane == 0) atomicAdd(a.n + i, w);
             }
-            // end of the segment: add this warp's 32 rows x its column slice into S, 16 columns
-            // at a time: the warp lays a 32 x 16 box out in shared memory (lane = row) and one TMA
+            // end of the item: add this warp's 32 rows x its column slice into S, 16 columns at a
+            // time: the warp lays a 32 x 16 box out in shared memory (lane = row) and one TMA
             // reduction adds it into S; rows and columns outside S are dropped by the hardware
-            const int tm = tile / a.ntn, tn = tile % a.ntn;
-            const int m0 = tm * DR_BM + (int)q * 32;
-            const int n_base = tn * DR_BN + c_begin * 16;
+            const DirectLayerMeta& lm = a.meta[it.layer];
+            const int m0 = it.tm * Cfg::TILE_M + (int)rank * DR_BM + (int)q * 32;
+            const int n_base = it.tn * DR_BN + c_begin * 16;
             const uint32_t box = staging_base + (uint32_t)(warp - 2) * DR_BOX_OUT;
             const uint32_t row_addr = box + (uint32_t)lane * 64u;
-            const bool flush = ok && a.S != nullptr && m0 < a.d_out;     // uniform across the warp
+            const bool flush = ok && lm.S != nullptr && m0 < lm.d_out;     // uniform across the warp
 #pragma unroll
             for (int cc = 0; cc < DR_CHUNKS_MAX; ++cc) {
-                if (flush && cc < n_chunks && n_base + cc * 16 < a.d_in) {
+                if (flush && cc < n_chunks && n_base + cc * 16 < lm.d_in) {
                     if (lane == 0) bulk_wait_read_all();                 // the previous box has been read
                     __syncwarp();
 #pragma unroll
@@ -897,7 +1053,7 @@ direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_reduce_add_2d(&tmS, box, n_base + cc * 16, m0);
+                        tma_reduce_add_2d(&a.maps[it.layer].tmS, box, n_base + cc * 16, m0);
                         bulk_commit_group();
                     }
                 }
@@ -905,16 +1061,17 @@ direct_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 for (int e = 0; e < 16; ++e) sacc[cc * 16 + e] = 0.f;
             }
         }
-        }
         if (lane == 0) bulk_wait_all();   // this warp's reductions into S are complete
         __syncwarp();
     }
 
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();   // neither CTA frees tensor memory or leaves while its peer still works
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 512);
+        if constexpr (PAIR) tmem_dealloc_pair(tmem_base, 512);
+        else tmem_dealloc(tmem_base, 512);
     }
     if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
 }
@@ -978,12 +1135,70 @@ static int make_map_f32(adloco_ctx* ctx, CUtensorMap* m, float* base, int64_t ro
     return ADLOCO_OK;
 }
 
+// Encoded tensor maps are kept per context, keyed by what determines them (base pointer,
+// extents, box, element type), so a layer that comes back every micro-batch is encoded once.
+struct MapKey {
+    const void* base;
+    int64_t e0, e1, e2;
+    uint32_t box, f32;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && e0 == o.e0 && e1 == o.e1 && e2 == o.e2 && box == o.box && f32 == o.f32;
+    }
+};
+struct MapKeyHash {
+    size_t operator()(const MapKey& k) const {
+        uint64_t h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
+        for (uint64_t v : {(uint64_t)k.e0, (uint64_t)k.e1, (uint64_t)k.e2, (uint64_t)k.box, (uint64_t)k.f32})
+            h = (h ^ v) * 0x100000001B3ull + (h >> 29);
+        return (size_t)h;
+    }
+};
+struct MapCache {
+    std::mutex mutex;
+    std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
+};
+constexpr size_t kMapCacheLimit = 8192;   // entries; beyond it the cache starts over
+
+static MapCache* map_cache(adloco_ctx* ctx) {
+    static std::mutex create_mutex;
+    std::lock_guard<std::mutex> lock(create_mutex);
+    if (!ctx->tensor_maps) ctx->tensor_maps = new (std::nothrow) MapCache();
+    return static_cast<MapCache*>(ctx->tensor_maps);
+}
+void free_tensor_map_cache(adloco_ctx* ctx) {
+    delete static_cast<MapCache*>(ctx->tensor_maps);
+    ctx->tensor_maps = nullptr;
+}
+
+template <typename Encode>
+static int cached_lookup(adloco_ctx* ctx, const MapKey& key, CUtensorMap* out, Encode encode) {
+    MapCache* c = map_cache(ctx);
+    if (!c) return encode(out);
+    std::lock_guard<std::mutex> lock(c->mutex);
+    auto it = c->maps.find(key);
+    if (it != c->maps.end()) { *out = it->second; return ADLOCO_OK; }
+    const int rc = encode(out);
+    if (rc != ADLOCO_OK) return rc;
+    if (c->maps.size() >= kMapCacheLimit) c->maps.clear();
+    c->maps.emplace(key, *out);
+    return ADLOCO_OK;
+}
+static int cached_map(adloco_ctx* ctx, CUtensorMap* m, const void* base, int64_t B, int64_t T, int64_t d,
+                      uint32_t box_tokens) {
+    const MapKey key{base, B, T, d, box_tokens, 0u};
+    return cached_lookup(ctx, key, m, [&](CUtensorMap* out) { return make_map(ctx, out, base, B, T, d, box_tokens); });
+}
+static int cached_map_f32(adloco_ctx* ctx, CUtensorMap* m, float* base, int64_t rows, int64_t cols, uint32_t box_cols) {
+    const MapKey key{base, rows, cols, 0, box_cols, 1u};
+    return cached_lookup(ctx, key, m, [&](CUtensorMap* out) { return make_map_f32(ctx, out, base, rows, cols, box_cols); });
+}
+
 int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                        int64_t d_out, float* n, int accumulate_norms, cudaStream_t st) {
     CUtensorMap tmX, tmD;
-    int rc = make_map(ctx, &tmX, X, B, T, d_in, GR_TILE);
+    int rc = cached_map(ctx, &tmX, X, B, T, d_in, GR_TILE);
     if (rc != ADLOCO_OK) return rc;
-    rc = make_map(ctx, &tmD, D, B, T, d_out, GR_TILE);
+    rc = cached_map(ctx, &tmD, D, B, T, d_out, GR_TILE);
     if (rc != ADLOCO_OK) return rc;
     GramArgs a;
     a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
@@ -1013,7 +1228,7 @@ int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
 int launch_embedding(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, int64_t T, int64_t d, int64_t V,
                      float* n, int accumulate_norms, float* S, int accumulate_sum, cudaStream_t st) {
     CUtensorMap tmD;
-    int rc = make_map(ctx, &tmD, D, B, T, d, GR_TILE);
+    int rc = cached_map(ctx, &tmD, D, B, T, d, GR_TILE);
     if (rc != ADLOCO_OK) return rc;
     EmbedArgs ea;
     GramArgs& a = ea.g;
@@ -1057,12 +1272,12 @@ int launch_embedding(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, 
 int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                      int64_t d_out, float* S, int accumulate_sum, cudaStream_t st) {
     CUtensorMap tmX, tmD;
-    int rc = make_map(ctx, &tmX, X, B, T, d_in, MG_BK);
+    int rc = cached_map(ctx, &tmX, X, B, T, d_in, MG_BK);
     if (rc != ADLOCO_OK) return rc;
-    rc = make_map(ctx, &tmD, D, B, T, d_out, MG_BK);
+    rc = cached_map(ctx, &tmD, D, B, T, d_out, MG_BK);
     if (rc != ADLOCO_OK) return rc;
     CUtensorMap tmS;
-    rc = make_map_f32(ctx, &tmS, S, d_out, d_in, 32);
+    rc = cached_map_f32(ctx, &tmS, S, d_out, d_in, 32);
     if (rc != ADLOCO_OK) return rc;
     MeanGradArgs a;
     a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
@@ -1085,42 +1300,120 @@ int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
     return ADLOCO_OK;
 }
 
-int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
-                         int64_t d_out, float* n, int accumulate_norms, float* S, int accumulate_sum,
-                         cudaStream_t st) {
-    CUtensorMap tmX, tmD;
-    int rc = make_map(ctx, &tmX, X, B, T, d_in, DR_BK);
-    if (rc != ADLOCO_OK) return rc;
-    rc = make_map(ctx, &tmD, D, B, T, d_out, DR_BK);
-    if (rc != ADLOCO_OK) return rc;
-    CUtensorMap tmS;
-    if (S) {
-        rc = make_map_f32(ctx, &tmS, S, d_out, d_in, 16);
-        if (rc != ADLOCO_OK) return rc;
-    } else {
-        tmS = tmX;   // never used by the kernel when S is null
+// Samples per work item: the count that minimises the busiest worker's units
+// (rounds of the round-robin deal x samples per item, plus a little per item for the
+// flush of the S tile), capped so that the chunks of samples the workers walk through at
+// any one time stay resident in L2.
+static int choose_chunk(int64_t total_tiles, int64_t B, int workers) {
+    int best = 1;
+    double best_cost = 1e300;
+    const int64_t cap = B < 4 ? B : 4;
+    for (int64_t c = 1; c <= cap; ++c) {
+        const int64_t items = total_tiles * ((B + c - 1) / c);
+        const int64_t rounds = (items + workers - 1) / workers;
+        const double cost = (double)rounds * ((double)c + 0.25);
+        if (cost <= best_cost) { best_cost = cost; best = (int)c; }
     }
-    DirectArgs a;
-    a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
-    a.ntm = (int)((d_out + DR_BM - 1) / DR_BM);
-    a.ntn = (int)((d_in + DR_BN - 1) / DR_BN);
-    if ((int64_t)a.ntm * a.ntn * B > 0x3fffffff) return ADLOCO_ERR_UNSUPPORTED;
-    const SplitPlan sp = make_split((int64_t)a.ntm * a.ntn, B, ctx->sm_count);
-    a.splits = sp.splits; a.chunk = sp.chunk; a.items = sp.items;
-    a.n = n; a.S = S; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
-    if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
-    if (S && !accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)d_out * (size_t)d_in * sizeof(float), st));
+    return best;
+}
+
+template <int CAP, bool PAIR>
+static int launch_direct_group_t(adloco_ctx* ctx, const adloco_linear_layer* layers, int n_layers, int64_t B, int64_t T,
+                                 float* n, cudaStream_t st) {
+    using Cfg = DirectCfg<PAIR>;
+    static DirectGroupArgs<CAP> a;             // 20 KB for CAP = 48: kept off the stack
+    static std::mutex args_mutex;              // the staging copy above is shared by all callers
+    std::lock_guard<std::mutex> lock(args_mutex);
+    const int workers = PAIR ? ctx->sm_count / 2 : ctx->sm_count;
+    int64_t total_tiles = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const int64_t ntm = (layers[l].d_out + Cfg::TILE_M - 1) / Cfg::TILE_M;
+        const int64_t ntn = (layers[l].d_in + DR_BN - 1) / DR_BN;
+        total_tiles += ntm * ntn;
+    }
+    const int chunk = choose_chunk(total_tiles, B, workers);
+    const int64_t n_chunks = (B + chunk - 1) / chunk;
+    if (total_tiles * n_chunks > 0x3fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    int item = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const adloco_linear_layer& L = layers[l];
+        int rc = cached_map(ctx, &a.maps[l].tmX, L.X, B, T, L.d_in, DR_BK);
+        if (rc != ADLOCO_OK) return rc;
+        rc = cached_map(ctx, &a.maps[l].tmD, L.D, B, T, L.d_out, DR_BK);
+        if (rc != ADLOCO_OK) return rc;
+        if (L.grad_sum) {
+            rc = cached_map_f32(ctx, &a.maps[l].tmS, L.grad_sum, L.d_out, L.d_in, 16);
+            if (rc != ADLOCO_OK) return rc;
+        } else {
+            a.maps[l].tmS = a.maps[l].tmX;   // never used by the kernel when S is null
+        }
+        DirectLayerMeta& m = a.meta[l];
+        m.S = L.grad_sum;
+        m.d_in = (int)L.d_in; m.d_out = (int)L.d_out;
+        m.ntn = (int)((L.d_in + DR_BN - 1) / DR_BN);
+        m.tiles = (int)((L.d_out + Cfg::TILE_M - 1) / Cfg::TILE_M) * m.ntn;
+        m.item_begin = item;
+        m.pad = 0;
+        item += m.tiles * (int)n_chunks;
+    }
+    a.n_layers = n_layers; a.B = (int)B; a.T = (int)T; a.kt = (int)((T + DR_BK - 1) / DR_BK);
+    a.chunk = chunk; a.total_items = item;
+    a.n = n; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
+    // every launch gets a work counter of its own from a small pool, so that launches on several
+    // streams do not share one
+    a.counter = ctx->sched_counters + (ctx->sched_next.fetch_add(1) % kSchedCounters);
+    ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(a.counter, 0, sizeof(int), st));
+    auto kern = direct_group_kernel<CAP, PAIR>;
     static std::atomic<bool> attr_set[64];   // the attribute is per device
     if (!attr_set[ctx->device & 63].load()) {
-        ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(direct_sqnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_SMEM));
+        ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
         attr_set[ctx->device & 63].store(true);
     }
-    const int grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
-    direct_sqnorm_kernel<<<grid, DR_THREADS, DR_SMEM, st>>>(tmX, tmD, tmS, a);
-    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    const int grid_workers = item < workers ? item : workers;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(PAIR ? 2 * grid_workers : grid_workers));
+    cfg.blockDim = dim3(DR_THREADS);
+    cfg.dynamicSmemBytes = Cfg::SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (PAIR) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    ADLOCO_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, kern, a));
     ctx->launches++;
     return ADLOCO_OK;
 }
 
+int launch_direct_group(adloco_ctx* ctx, const adloco_linear_layer* layers, int n_layers, int64_t B, int64_t T,
+                        float* n, int accumulate_norms, int accumulate_sum, int pair, cudaStream_t st) {
+    if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
+    if (!accumulate_sum)
+        for (int l = 0; l < n_layers; ++l)
+            if (layers[l].grad_sum)
+                ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(layers[l].grad_sum, 0,
+                                                     (size_t)layers[l].d_out * (size_t)layers[l].d_in * sizeof(float), st));
+    // as many layers per launch as the kernel's argument block holds
+    for (int l0 = 0; l0 < n_layers; l0 += kDirectGroupCap) {
+        const int nl = n_layers - l0 < kDirectGroupCap ? n_layers - l0 : kDirectGroupCap;
+        int rc;
+        if (nl == 1) rc = pair ? launch_direct_group_t<1, true>(ctx, layers + l0, 1, B, T, n, st)
+                               : launch_direct_group_t<1, false>(ctx, layers + l0, 1, B, T, n, st);
+        else rc = pair ? launch_direct_group_t<kDirectGroupCap, true>(ctx, layers + l0, nl, B, T, n, st)
+                       : launch_direct_group_t<kDirectGroupCap, false>(ctx, layers + l0, nl, B, T, n, st);
+        if (rc != ADLOCO_OK) return rc;
+    }
+    return ADLOCO_OK;
+}
+
+int launch_direct_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                         int64_t d_out, float* n, int accumulate_norms, float* S, int accumulate_sum, int pair,
+                         cudaStream_t st) {
+    adloco_linear_layer L;
+    L.X = X; L.D = D; L.d_in = d_in; L.d_out = d_out; L.grad_sum = S;
+    return launch_direct_group(ctx, &L, 1, B, T, n, accumulate_norms, accumulate_sum, pair, st);
+}
 
 }  // namespace adloco

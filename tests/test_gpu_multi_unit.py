@@ -56,13 +56,13 @@ MULTI_UNIT_SHAPES = [
 
 
 @pytest.mark.parametrize("B,T,d_in,d_out", MULTI_UNIT_SHAPES)
-@pytest.mark.parametrize("method", ["direct", "gram"])
+@pytest.mark.parametrize("method", ["direct", "pair", "gram"])
 def test_ctas_with_several_units_match_the_oracle(ctx, B, T, d_in, d_out, method):
     X, D = W.linear_layer(B, T, d_in, d_out, seed=7 * B + T, device=DEV)
     _check_layer(ctx, X, D, method, f"{method} B={B} T={T} {d_in}->{d_out}")
 
 
-@pytest.mark.parametrize("method", ["direct", "gram"])
+@pytest.mark.parametrize("method", ["direct", "pair", "gram"])
 def test_several_units_exact_on_integers(ctx, method):
     # T = 16 keeps every entry of a per-sample gradient below 2^8 and every sum below 2^24: exact in fp32
     X, D = W.small_integer_layer(11, 16, 768, 1536, seed=5, device=DEV)
@@ -72,13 +72,14 @@ def test_several_units_exact_on_integers(ctx, method):
     torch.cuda.synchronize()
     n_ref, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
     assert np.array_equal(S.cpu().numpy().astype(np.float64), S_ref)
-    assert np.allclose(n.cpu().numpy(), n_ref, rtol=1e-6)      # n_i ~ 1e8 exceeds 2^24: rounded, not exact
+    assert np.allclose(n.cpu().numpy(), n_ref, rtol=1e-5)      # n_i ~ 3e8 exceeds 2^24: hundreds of fp32 adds, each rounded
 
 
 def test_config3_layer_direct_route_full_size(ctx):
     """B=32, T=1024, 768 -> 3072 by the direct route: 72 tiles x 2 chunks of 16 samples."""
     X, D = W.linear_layer(32, 1024, 768, 3072, seed=3, device=DEV)
     _check_layer(ctx, X, D, "direct", "config 3 direct")
+    _check_layer(ctx, X, D, "pair", "config 3 pair")
     _check_layer(ctx, X, D, "auto", "config 3 auto")
 
 
@@ -104,3 +105,61 @@ def test_embedding_with_several_items_per_cta(ctx):
     torch.cuda.synchronize()
     n_ref2, _ = O.embedding_terms(ids2.cpu().numpy(), W.to_numpy(D), V)
     assert np.allclose(n.cpu().numpy(), n_ref2, rtol=TOL_BF16)
+
+
+# ---------------------------------------------------------------- groups of layers in one launch
+def _group_case(ctx, shapes, B, T, method, seed, accumulate=False):
+    data = [W.linear_layer(B, T, di, do, seed=seed + l, device=DEV) for l, (di, do) in enumerate(shapes)]
+    sums = [torch.full((do, di), 2.0 if accumulate else -7.0, device=DEV) if (l % 5) != 3 else None
+            for l, (di, do) in enumerate(shapes)]                       # some layers give no sum buffer
+    n = torch.full((B,), 1.0 if accumulate else -7.0, device=DEV)
+    ctx.linear_sqnorm_group([(X, D, S) for (X, D), S in zip(data, sums)], n, method=method,
+                            accumulate_norms=accumulate, accumulate_sum=accumulate)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    n_ref = np.zeros(B)
+    for (X, D), S in zip(data, sums):
+        n_l, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
+        n_ref += n_l
+        if S is not None:
+            got = S.cpu().numpy() - (2.0 if accumulate else 0.0)
+            assert np.allclose(got, S_ref, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(S_ref).max() * 0.05 + (1e-5 if accumulate else 0))
+    got_n = n.cpu().numpy() - (1.0 if accumulate else 0.0)
+    assert np.allclose(got_n, n_ref, rtol=TOL_BF16, atol=1e-4 if accumulate else 0), (method, got_n / n_ref)
+
+
+@pytest.mark.parametrize("method", ["direct", "pair", "auto"])
+def test_group_of_layers_matches_the_oracle(ctx, method):
+    """One launch over layers of unlike shapes: the per-sample norms add up over the layers, every
+    layer's gradient sum lands in its own buffer; ragged widths, a layer narrower than one tile,
+    a transformer block's four shapes (scaled down), layers without a sum buffer."""
+    shapes = [(256, 768), (256, 256), (256, 1024), (1024, 256), (72, 40), (8, 8), (520, 136), (136, 520)]
+    _group_case(ctx, shapes, B=6, T=200, method=method, seed=300)
+    _group_case(ctx, shapes[:3], B=2, T=64, method=method, seed=400, accumulate=True)
+
+
+@pytest.mark.parametrize("method", ["direct", "pair"])
+def test_group_longer_than_one_launch_holds(ctx, method):
+    # 53 layers: the argument block of one launch holds 48, so the call is split in two
+    shapes = [(64 + 8 * (l % 5), 32 + 16 * (l % 7)) for l in range(53)]
+    _group_case(ctx, shapes, B=3, T=96, method=method, seed=500)
+
+
+def test_group_of_one_block_at_full_size(ctx):
+    """The four linear layers of a GPT-2-small block, B=32, T=1024, as one group by the
+    automatic route: about 2000 work items of four samples over the SMs."""
+    shapes = list(W.GPT2_SMALL_BLOCK_LINEARS)
+    _group_case(ctx, shapes, B=32, T=1024, method="auto", seed=600)
+
+
+def test_group_argument_errors(ctx):
+    X, D = W.linear_layer(2, 64, 64, 64, seed=1, device=DEV)
+    n = torch.zeros(2, device=DEV)
+    before = ctx.launch_count
+    with pytest.raises(A.AdlocoError) as e:
+        ctx.linear_sqnorm_group([(X, D, None)], n, method="gram")          # the group call has no Gram route
+    assert e.value.status == A.ERR_INVALID_ARG
+    X2, D2 = W.linear_layer(2, 64, 12, 64, seed=1, device=DEV)
+    with pytest.raises(A.AdlocoError) as e:
+        ctx.linear_sqnorm_group([(X, D, None), (X2, D2, None)], n)         # d_in = 12 is not a multiple of 8
+    assert e.value.status == A.ERR_UNSUPPORTED and ctx.launch_count == before

@@ -52,7 +52,7 @@ def test_single_process_is_the_identity():
     assert ab["nt2"] == 4 * 64 * (1 << 24) and ab["os2"] == (2 * 8 + 16) * 124_439_808
     assert ab["os5"] == (2 * 4 + 16) * 1_300_000_000 and ab["acc5"] == 8 * (4 * 32 + 8) * (1 << 22)
     flops, launches = bench.model_flops()
-    assert launches == 192 and flops == 4 * 12 * 2 * 32 * 1024 * (768 * 2304 + 768 * 768 + 2 * 768 * 3072)
+    assert launches == 4 and flops == 4 * 12 * 2 * 32 * 1024 * (768 * 2304 + 768 * 768 + 2 * 768 * 3072)
 
 
 def test_shard_bounds_partition_the_vector():
