@@ -329,6 +329,7 @@ int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
         return ADLOCO_ERR_INVALID_ARG;
     if (!ctx || !X || !D || !per_sample_sqnorm) return ADLOCO_ERR_INVALID_ARG;
     if (B < 1 || T < 1 || d_in < 1 || d_out < 1) return ADLOCO_ERR_INVALID_ARG;
+    const bool was_auto = (method == ADLOCO_LINEAR_AUTO);
     if (method == ADLOCO_LINEAR_AUTO) {
         // tensor work of the two routes at the granularity the kernels execute, divided by
         // the share of the SMs their work items can occupy (few tokens give the Gram kernel
@@ -353,6 +354,9 @@ int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
     if (!aligned16(X) || !aligned16(D)) return ADLOCO_ERR_ALIGNMENT;
     if (grad_sum && !aligned16(grad_sum)) return ADLOCO_ERR_ALIGNMENT;
     DeviceGuard g(ctx->device);
+    // the automatic route takes the CTA-pair form of the direct kernel where clusters can be launched
+    // and the tile is at least one pair's worth of rows
+    if (was_auto && method == ADLOCO_LINEAR_DIRECT && d_out > 128 && pair_launch_ok(ctx)) method = ADLOCO_LINEAR_DIRECT_PAIR;
     if (method == ADLOCO_LINEAR_DIRECT_PAIR && !pair_launch_ok(ctx)) return ADLOCO_ERR_UNSUPPORTED;
     return launch_direct_sqnorm(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, grad_sum,
                                 accumulate_sum, method == ADLOCO_LINEAR_DIRECT_PAIR, static_cast<cudaStream_t>(stream));
