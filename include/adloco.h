@@ -383,6 +383,30 @@ int adloco_outer_step_host(adloco_ctx* ctx, const void* const* inst_params_host,
                            int32_t K, int64_t P, float* theta_host, float* mom_host, float lr, float momentum,
                            int nesterov, void* stream);
 
+/* The outer step when every GPU holds ONE whole instance (and the shared starting point
+ * theta) but only a slice of the momentum: the K pseudo-gradients are summed across the
+ * GPUs by one reduce-scatter -- the single communication of the method (last loop of
+ * Algorithm 3: the workers' differences are gathered and averaged) -- which the caller
+ * performs between these calls, with whatever collective library it uses:
+ *   1. adloco_pseudo_gradient    pseudo_grad = theta - theta_k, fp32 [P]      (every rank)
+ *   2. reduce-scatter (sum) of pseudo_grad over the K ranks -> pseudo_grad_sum, this rank's slice
+ *   3. adloco_outer_apply        d = pseudo_grad_sum / K; v' = momentum v + d;
+ *                                u = d + momentum v' | v'; theta' = theta - lr u   (on the slice)
+ *   4. all-gather of the theta' slices, then adloco_refresh_instance: theta_k = theta'
+ *      rounded to the instance type (Algorithm 3 restarts every worker from theta).
+ * All pointers dev, 16-byte aligned; theta/mom in and out may alias exactly.  The update is
+ * carried in fp64 and rounded once, as in adloco_outer_step.  The K terms cross the exchange
+ * as fp32 and are summed by the collective in fp32: against adloco_outer_step (which sums
+ * them in fp64) the sum can be off by up to (K - 1/2) ulp of sum_k |theta - theta_k|, which
+ * shows where the terms cancel and the update itself is small. */
+int adloco_pseudo_gradient(adloco_ctx* ctx, const float* theta, const void* inst_params, adloco_dtype inst_dtype,
+                           int64_t P, float* pseudo_grad, void* stream);
+int adloco_outer_apply(adloco_ctx* ctx, const float* pseudo_grad_sum, int32_t K, int64_t P, const float* theta_in,
+                       float* theta_out, const float* mom_in, float* mom_out, float lr, float momentum, int nesterov,
+                       void* stream);
+int adloco_refresh_instance(adloco_ctx* ctx, const float* theta, void* inst_params, adloco_dtype inst_dtype, int64_t P,
+                            void* stream);
+
 /* ---- trainer merge --------------------------------------------------------- */
 
 /* CheckMerge (Algorithm 1), host only: writes into merge_idx (host, capacity >= w)

@@ -26,6 +26,7 @@ EXPORTS = (
     "adloco_norm_test", "adloco_test_decide", "adloco_norm_test_host", "adloco_norm_test_noalloc", "adloco_inner_product_test", "adloco_gram_sqnorm", "adloco_linear_sqnorm", "adloco_linear_sqnorm_group", "adloco_vector_param_sqnorm", "adloco_embedding_sqnorm",
     "adloco_accum_create", "adloco_accum_reset", "adloco_accum_destroy", "adloco_accumulate",
     "adloco_accum_finalize", "adloco_outer_step", "adloco_outer_step_host", "adloco_check_merge", "adloco_merge",
+    "adloco_pseudo_gradient", "adloco_outer_apply", "adloco_refresh_instance",
 )
 
 
@@ -115,6 +116,9 @@ def load_library() -> C.CDLL:
         "adloco_outer_step": (C.c_int, [vp, C.POINTER(vp), C.c_int, i32, i64, vp, vp, vp, vp, f32, f32, C.c_int,
                                         C.POINTER(vp), vp]),
         "adloco_outer_step_host": (C.c_int, [vp, C.POINTER(vp), C.c_int, i32, i64, vp, vp, f32, f32, C.c_int, vp]),
+        "adloco_pseudo_gradient": (C.c_int, [vp, vp, vp, C.c_int, i64, vp, vp]),
+        "adloco_outer_apply": (C.c_int, [vp, vp, i32, i64, vp, vp, vp, vp, f32, f32, C.c_int, vp]),
+        "adloco_refresh_instance": (C.c_int, [vp, vp, vp, C.c_int, i64, vp]),
         "adloco_check_merge": (C.c_int, [C.POINTER(i64), i32, i32, C.POINTER(i32)]),
         "adloco_merge": (C.c_int, [vp, C.POINTER(vp), C.POINTER(i64), C.c_int, i32, i64, vp, C.POINTER(i32), vp]),
     }
@@ -350,6 +354,26 @@ class Context:
                                              theta_host.numel(), _ptr(theta_host), _ptr(mom_host), float(lr),
                                              float(momentum), int(bool(nesterov)), _stream(stream))
         self.check(rc, "adloco_outer_step_host")
+
+    # ------------------------------------------------------------------ outer step around an exchange
+    def pseudo_gradient(self, theta, instance, out, *, stream=None):
+        """adloco_pseudo_gradient: out = theta - instance (fp32 [P])."""
+        rc = self.lib.adloco_pseudo_gradient(self.h, _ptr(theta), _ptr(instance), _dtype_code(instance.dtype),
+                                             theta.numel(), _ptr(out), _stream(stream))
+        self.check(rc, "adloco_pseudo_gradient")
+
+    def outer_apply(self, pseudo_grad_sum, K, theta, mom, *, lr, momentum, nesterov=True, stream=None):
+        """adloco_outer_apply, in place on the slices theta and mom."""
+        rc = self.lib.adloco_outer_apply(self.h, _ptr(pseudo_grad_sum), int(K), theta.numel(), _ptr(theta), _ptr(theta),
+                                         _ptr(mom), _ptr(mom), float(lr), float(momentum), int(bool(nesterov)),
+                                         _stream(stream))
+        self.check(rc, "adloco_outer_apply")
+
+    def refresh_instance(self, theta, instance, *, stream=None):
+        """adloco_refresh_instance: instance = theta rounded to the instance's type."""
+        rc = self.lib.adloco_refresh_instance(self.h, _ptr(theta), _ptr(instance), _dtype_code(instance.dtype),
+                                              theta.numel(), _stream(stream))
+        self.check(rc, "adloco_refresh_instance")
 
     # ------------------------------------------------------------------ merge
     def merge(self, members, weights, out, *, stream=None) -> int:

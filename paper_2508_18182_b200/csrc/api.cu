@@ -588,6 +588,42 @@ int adloco_outer_step_host(adloco_ctx* ctx, const void* const* inst_params_host,
 }
 
 // ---------------------------------------------------------------------------------
+// outer step split around an exchange of pseudo-gradients
+// ---------------------------------------------------------------------------------
+int adloco_pseudo_gradient(adloco_ctx* ctx, const float* theta, const void* inst_params, adloco_dtype inst_dtype,
+                           int64_t P, float* pseudo_grad, void* stream) {
+    if (!ctx || !theta || !inst_params || !pseudo_grad || P < 1) return ADLOCO_ERR_INVALID_ARG;
+    if (inst_dtype != ADLOCO_F32 && inst_dtype != ADLOCO_BF16) return ADLOCO_ERR_INVALID_ARG;
+    if (!aligned16(theta) || !aligned16(inst_params) || !aligned16(pseudo_grad)) return ADLOCO_ERR_ALIGNMENT;
+    DeviceGuard g(ctx->device);
+    return launch_pseudo_grad(ctx, theta, inst_params, inst_dtype == ADLOCO_BF16, pseudo_grad, P,
+                              static_cast<cudaStream_t>(stream));
+}
+
+int adloco_outer_apply(adloco_ctx* ctx, const float* pseudo_grad_sum, int32_t K, int64_t P, const float* theta_in,
+                       float* theta_out, const float* mom_in, float* mom_out, float lr, float momentum, int nesterov,
+                       void* stream) {
+    if (!ctx || !pseudo_grad_sum || !theta_in || !theta_out || !mom_in || !mom_out || K < 1 || P < 1)
+        return ADLOCO_ERR_INVALID_ARG;
+    if (!(lr == lr) || !(momentum == momentum)) return ADLOCO_ERR_INVALID_ARG;
+    if (!aligned16(pseudo_grad_sum) || !aligned16(theta_in) || !aligned16(theta_out) || !aligned16(mom_in) ||
+        !aligned16(mom_out))
+        return ADLOCO_ERR_ALIGNMENT;
+    DeviceGuard g(ctx->device);
+    return launch_outer_apply(ctx, pseudo_grad_sum, K, P, theta_in, theta_out, mom_in, mom_out, lr, momentum,
+                              nesterov ? 1 : 0, static_cast<cudaStream_t>(stream));
+}
+
+int adloco_refresh_instance(adloco_ctx* ctx, const float* theta, void* inst_params, adloco_dtype inst_dtype, int64_t P,
+                            void* stream) {
+    if (!ctx || !theta || !inst_params || P < 1) return ADLOCO_ERR_INVALID_ARG;
+    if (inst_dtype != ADLOCO_F32 && inst_dtype != ADLOCO_BF16) return ADLOCO_ERR_INVALID_ARG;
+    if (!aligned16(theta) || !aligned16(inst_params)) return ADLOCO_ERR_ALIGNMENT;
+    DeviceGuard g(ctx->device);
+    return launch_refresh(ctx, theta, inst_params, inst_dtype == ADLOCO_BF16, P, static_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------------------------
 // trainer merge
 // ---------------------------------------------------------------------------------
 int adloco_check_merge(const int64_t* b_req, int32_t k, int32_t w, int32_t* merge_idx) {

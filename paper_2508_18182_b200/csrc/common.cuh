@@ -142,6 +142,11 @@ struct OuterLaunch {
 };
 int launch_outer_step(adloco_ctx* ctx, const OuterLaunch& l, cudaStream_t st);
 
+int launch_pseudo_grad(adloco_ctx* ctx, const float* theta, const void* inst, int bf16, float* g, int64_t P, cudaStream_t st);
+int launch_outer_apply(adloco_ctx* ctx, const float* g_sum, int K, int64_t P, const float* th_in, float* th_out,
+                       const float* v_in, float* v_out, float lr, float mu, int nesterov, cudaStream_t st);
+int launch_refresh(adloco_ctx* ctx, const float* theta, void* inst, int bf16, int64_t P, cudaStream_t st);
+
 struct MergeLaunch {
     const void* x[kMaxInstances];
     float coef[kMaxInstances];

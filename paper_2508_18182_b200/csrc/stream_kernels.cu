@@ -253,6 +253,9 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
 
         float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
         float4 sd = c, sdd = c;
+        // switch mode: the sums so far are fetched now, so that their latency hides behind the rows
+        float4 so = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (a.mode == NT_MICRO && nvalid > 0) so = load4<VEC>(a.S + col, nvalid);
         for (int64_t i0 = 0; i0 < B; i0 += RB) {
 #pragma unroll
             for (int r0 = 0; r0 < RB; r0 += CH) {
@@ -293,8 +296,6 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
         f_css += (sdd.x - sd.x * sd.x * invB) + (sdd.y - sd.y * sd.y * invB) +
                  (sdd.z - sd.z * sd.z * invB) + (sdd.w - sd.w * sd.w * invB);
         if (a.mode == NT_MICRO) {
-            float4 so = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (nvalid > 0) so = load4<VEC>(a.S + col, nvalid);
             // pairwise (Chan) update of the centred sum of squares needs ||mean_mb - mean_prev||^2
             const float ex = s.x * invB - so.x * inv_cprev, ey = s.y * invB - so.y * inv_cprev;
             const float ez = s.z * invB - so.z * inv_cprev, ew = s.w * invB - so.w * inv_cprev;
@@ -1047,6 +1048,114 @@ int launch_outer_step(adloco_ctx* ctx, const OuterLaunch& l, cudaStream_t st) {
         else { if (l.has_wb) ADLOCO_OUTER_LAUNCH(false, true, 4); else ADLOCO_OUTER_LAUNCH(false, false, 4); }
     }
 #undef ADLOCO_OUTER_LAUNCH
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+// ---------------------------------------------------------------------------------
+// outer step with an exchange: each GPU holds one whole instance and a slice of v
+// ---------------------------------------------------------------------------------
+// Three elementwise passes around the one exchange of the pseudo-gradients:
+//   pseudo_grad_kernel   g = theta - x_k                  (this rank's term of the sum)
+//   [the K terms are summed slice-wise across the ranks by a reduce-scatter]
+//   outer_apply_kernel   d = g_sum / K, then the same update as outer_step_kernel
+//   refresh_kernel       x_k = theta' (cast to the instance type) once theta' is gathered
+template <bool BF16>
+__global__ void __launch_bounds__(256) pseudo_grad_kernel(const float* __restrict__ theta, const void* __restrict__ inst,
+                                                           float* __restrict__ g, int64_t P) {
+    const int64_t nvec = P / 4;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
+        const float4 t = __ldcs(reinterpret_cast<const float4*>(theta) + i);
+        float x[4];
+        load_inst4<BF16>(inst, i, x);
+        __stcs(reinterpret_cast<float4*>(g) + i, make_float4(t.x - x[0], t.y - x[1], t.z - x[2], t.w - x[3]));
+    }
+    if (blockIdx.x == 0) {
+        for (int64_t j = nvec * 4 + threadIdx.x; j < P; j += blockDim.x) {
+            float x;
+            if (BF16) x = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(inst)[j]);
+            else x = reinterpret_cast<const float*>(inst)[j];
+            g[j] = theta[j] - x;
+        }
+    }
+}
+
+struct ApplyArgs {
+    const float* g_sum;
+    const float* th_in;
+    float* th_out;
+    const float* v_in;
+    float* v_out;
+    int64_t P;
+    OuterArgs u;      // invK, lr, mu, nesterov (the instance pointers are unused)
+};
+
+__global__ void __launch_bounds__(256) outer_apply_kernel(const __grid_constant__ ApplyArgs a) {
+    const int64_t nvec = a.P / 4;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
+        const float4 g4 = __ldcs(reinterpret_cast<const float4*>(a.g_sum) + i);
+        const float4 t4 = __ldcs(reinterpret_cast<const float4*>(a.th_in) + i);
+        const float4 v4 = __ldcs(reinterpret_cast<const float4*>(a.v_in) + i);
+        const float g[4] = {g4.x, g4.y, g4.z, g4.w}, th[4] = {t4.x, t4.y, t4.z, t4.w}, v[4] = {v4.x, v4.y, v4.z, v4.w};
+        float tn[4], vn[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) outer_update(th[e], v[e], (double)g[e], a.u, tn[e], vn[e]);
+        __stcs(reinterpret_cast<float4*>(a.th_out) + i, make_float4(tn[0], tn[1], tn[2], tn[3]));
+        __stcs(reinterpret_cast<float4*>(a.v_out) + i, make_float4(vn[0], vn[1], vn[2], vn[3]));
+    }
+    if (blockIdx.x == 0) {
+        for (int64_t j = nvec * 4 + threadIdx.x; j < a.P; j += blockDim.x) {
+            float tn, vn;
+            outer_update(a.th_in[j], a.v_in[j], (double)a.g_sum[j], a.u, tn, vn);
+            a.th_out[j] = tn;
+            a.v_out[j] = vn;
+        }
+    }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(256) refresh_kernel(const float* __restrict__ theta, void* __restrict__ inst, int64_t P) {
+    const int64_t nvec = P / 4;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
+        const float4 t = __ldcs(reinterpret_cast<const float4*>(theta) + i);
+        if (BF16) reinterpret_cast<uint2*>(inst)[i] = make_uint2(pack_bf16(t.x, t.y), pack_bf16(t.z, t.w));
+        else reinterpret_cast<float4*>(inst)[i] = t;
+    }
+    if (blockIdx.x == 0) {
+        for (int64_t j = nvec * 4 + threadIdx.x; j < P; j += blockDim.x) {
+            if (BF16) reinterpret_cast<__nv_bfloat16*>(inst)[j] = __float2bfloat16_rn(theta[j]);
+            else reinterpret_cast<float*>(inst)[j] = theta[j];
+        }
+    }
+}
+
+int launch_pseudo_grad(adloco_ctx* ctx, const float* theta, const void* inst, int bf16, float* g, int64_t P, cudaStream_t st) {
+    if (bf16) pseudo_grad_kernel<true><<<elementwise_grid(ctx, pseudo_grad_kernel<true>, P / 4, 256), 256, 0, st>>>(theta, inst, g, P);
+    else pseudo_grad_kernel<false><<<elementwise_grid(ctx, pseudo_grad_kernel<false>, P / 4, 256), 256, 0, st>>>(theta, inst, g, P);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+int launch_outer_apply(adloco_ctx* ctx, const float* g_sum, int K, int64_t P, const float* th_in, float* th_out,
+                       const float* v_in, float* v_out, float lr, float mu, int nesterov, cudaStream_t st) {
+    ApplyArgs a;
+    memset(&a, 0, sizeof(a));
+    a.g_sum = g_sum; a.th_in = th_in; a.th_out = th_out; a.v_in = v_in; a.v_out = v_out; a.P = P;
+    a.u.invK = 1.0 / (double)K; a.u.lr = lr; a.u.mu = mu; a.u.K = K; a.u.nesterov = nesterov;
+    outer_apply_kernel<<<elementwise_grid(ctx, outer_apply_kernel, P / 4, 256), 256, 0, st>>>(a);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+int launch_refresh(adloco_ctx* ctx, const float* theta, void* inst, int bf16, int64_t P, cudaStream_t st) {
+    if (bf16) refresh_kernel<true><<<elementwise_grid(ctx, refresh_kernel<true>, P / 4, 256), 256, 0, st>>>(theta, inst, P);
+    else refresh_kernel<false><<<elementwise_grid(ctx, refresh_kernel<false>, P / 4, 256), 256, 0, st>>>(theta, inst, P);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;

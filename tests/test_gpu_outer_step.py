@@ -141,3 +141,92 @@ def test_sharded_outer_step_equals_the_whole(ctx, world):
         covered = hi
     assert covered == theta.numel()
     assert torch.equal(th, th_ref) and torch.equal(v, v_ref)
+
+
+# ---------------------------------------------------------------- outer step split around an exchange
+@pytest.mark.parametrize("K,P,dtype", [(2, 100003, torch.bfloat16), (4, 65536, torch.float32), (3, 13, torch.bfloat16),
+                                       (4, 1 << 20, torch.bfloat16)])
+def test_exchange_form_matches_oracle(ctx, K, P, dtype):
+    """One instance per rank: pseudo-gradient kernel on every rank, the K terms summed slice-wise (here
+    by torch, standing in for the reduce-scatter between GPUs), update kernel on every slice, refresh.
+    Result against the oracle's outer step on the whole vector.  The terms theta - theta_k cross the
+    exchange as fp32 and are summed there in fp32, so beside the 2 ulp of the output rounding the result
+    carries their rounding: at most (K - 1/2) ulp of sum_k |theta - theta_k| on the sum, i.e. that / K on d
+    and v', times lr (1 + mu) on theta' -- visible where the K terms cancel and the update is small."""
+    from paper_2508_18182_b200.exchange import slice_length
+    theta, inst, mom = W.outer_state(K, P, inst_dtype=dtype, seed=91, device=DEV, zero_momentum=False)
+    th0, v0 = W.to_numpy(theta).astype(np.float64), W.to_numpy(mom).astype(np.float64)
+    inst_n = [W.to_numpy(t) for t in inst]
+    lr, mu = float(np.float32(0.7)), float(np.float32(0.9))
+    th_ref, v_ref = O.outer_step(W.to_numpy(theta), inst_n, W.to_numpy(mom), lr=lr, momentum=mu)
+    d = np.mean([th0 - O.widen(x) for x in inst_n], axis=0)
+    L = slice_length(P, K)
+    g = [torch.zeros(L * K, device=DEV) for _ in range(K)]
+    for k in range(K):
+        ctx.pseudo_gradient(theta, inst[k], g[k][:P])
+        ref = (th0 - O.widen(inst_n[k])).astype(np.float32)                  # each term, rounded to fp32 once
+        assert np.array_equal(g[k][:P].cpu().numpy(), ref)
+        assert not g[k][P:].any()
+    total = g[0].clone()
+    for k in range(1, K):
+        total += g[k]
+    th, v = theta.clone(), mom.clone()
+    for r in range(K):
+        lo, hi = min(P, r * L), min(P, r * L + L)
+        if hi > lo:
+            ctx.outer_apply(total[lo:hi], K, th[lo:hi], v[lo:hi], lr=0.7, momentum=0.9)
+    torch.cuda.synchronize()
+    from parity import ulp32
+    terms = np.sum([np.abs(th0 - O.widen(x)) for x in inst_n], axis=0)
+    exch = (K - 0.5) / K * ulp32(terms)
+    mag_t = np.maximum(np.maximum(np.abs(th0), np.abs(th_ref)), np.abs(th0 - th_ref))
+    mag_v = np.maximum(np.maximum(np.abs(v_ref), np.abs(mu * v0)), np.abs(d))
+    et = np.abs(th.cpu().numpy().astype(np.float64) - th_ref) / (2 * ulp32(mag_t) + lr * (1 + mu) * exch)
+    ev = np.abs(v.cpu().numpy().astype(np.float64) - v_ref) / (2 * ulp32(mag_v) + exch)
+    assert et.max() <= 1.0 and ev.max() <= 1.0, (K, P, float(et.max()), float(ev.max()))
+    # where no term needed rounding (theta and theta_k close: most elements) the fused kernel's 2 ulp hold
+    exact = np.all([(th0 - O.widen(x)).astype(np.float32).astype(np.float64) == th0 - O.widen(x) for x in inst_n], axis=0)
+    exact &= (sum(g[k][:P].double() for k in range(K)).cpu().numpy() == total[:P].cpu().numpy().astype(np.float64))
+    assert exact.mean() > 0.5 or K > 2
+    e2 = np.abs(th.cpu().numpy().astype(np.float64) - th_ref)[exact] / ulp32(mag_t)[exact]
+    assert e2.size == 0 or e2.max() <= 2.0
+    for k in range(K):
+        ctx.refresh_instance(th, inst[k])
+        assert torch.equal(inst[k], th.to(dtype))
+    with pytest.raises(A.AdlocoError) as e:
+        ctx.outer_apply(total[1:9], K, th[:8], v[:8], lr=0.7, momentum=0.9)   # misaligned sum buffer
+    assert e.value.status == A.ERR_ALIGNMENT
+
+
+def test_exchanged_outer_step_through_a_process_group_of_one():
+    """The same path through ExchangedOuterStep with a real process group on the GPU (one rank: the
+    reduce-scatter and the gather move the slice to itself) -- the NCCL plumbing and the buffers."""
+    import torch.distributed as dist
+    from paper_2508_18182_b200.exchange import ExchangedOuterStep, slice_length
+    import os
+    c = A.Context(0)
+    P = 30011
+    theta, inst, mom = W.outer_state(1, P, inst_dtype=torch.bfloat16, seed=17, device=DEV, zero_momentum=False)
+    lr, mu = float(np.float32(0.7)), float(np.float32(0.9))
+    th_ref, v_ref = O.outer_step(W.to_numpy(theta), [W.to_numpy(inst[0])], W.to_numpy(mom), lr=lr, momentum=mu)
+    th0, v0 = W.to_numpy(theta).astype(np.float64), W.to_numpy(mom).astype(np.float64)
+    d = th0 - O.widen(W.to_numpy(inst[0]))
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", str(29700 + os.getpid() % 200))
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device(DEV))
+    try:
+        L = slice_length(P, 1)
+        v_slice = torch.zeros(L, device=DEV)
+        v_slice[:P] = mom
+        state = ExchangedOuterStep(c, theta, inst[0], v_slice)
+        th = state.step(lr=0.7, momentum=0.9)
+        torch.cuda.synchronize()
+        from parity import ulp32
+        mag_t = np.maximum(np.maximum(np.abs(th0), np.abs(th_ref)), np.abs(th0 - th_ref))
+        et = np.abs(th.cpu().numpy().astype(np.float64) - th_ref) / (2 * ulp32(mag_t) + lr * (1 + mu) * 0.5 * ulp32(d))
+        ev = np.abs(state.mom[:P].cpu().numpy().astype(np.float64) - v_ref) / (2 * ulp32(np.maximum(np.abs(v_ref), np.abs(d))) + 0.5 * ulp32(d))
+        assert et.max() <= 1.0 and ev.max() <= 1.0, (float(et.max()), float(ev.max()))
+        assert torch.equal(state.instance, th.to(torch.bfloat16))
+    finally:
+        dist.destroy_process_group()
+        c.close()
