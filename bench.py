@@ -379,6 +379,7 @@ def run_ours(args, rank, world, local_rank):
     reps = 20
     g0, g1, g2, g3, g4, g5 = ev(), ev(), ev(), ev(), ev(), ev()
     torch.cuda.synchronize()
+    time.sleep(1.0)           # let the clocks recover from the timed region: these are burst figures
     g0.record(stream)
     for _ in range(reps):
         ctx.gram_sqnorm(X, D, n_layer)
@@ -396,6 +397,31 @@ def run_ours(args, rank, world, local_rank):
     g5.record(stream)
     torch.cuda.synchronize()
     gram_only_ms = g0.elapsed_time(g1) / reps
+    # the streaming kernels by themselves, after a pause that lets the clocks recover from the power cap
+    # the tensor-core sections of the step run into (the cap holds the SM clock, and with it the on-chip
+    # network, well below its maximum for the whole step)
+    time.sleep(1.0)
+    alone = {}
+
+    def time_alone(name, fn, n=20):
+        fn()
+        torch.cuda.synchronize()
+        a0, a1 = ev(), ev()
+        a0.record(stream)
+        for _ in range(n):
+            fn()
+        a1.record(stream)
+        torch.cuda.synchronize()
+        alone[name] = a0.elapsed_time(a1) / n
+
+    def acc5_only():
+        for mb in mbs5:
+            acc5.accumulate(mb)
+
+    time_alone("nt2", lambda: ctx.norm_test(G, params[0], sync=False))
+    time_alone("os2", lambda: ctx.outer_step(inst, theta, mom, lr=LR, momentum=MU, nesterov=True))
+    time_alone("os5", lambda: ctx.outer_step(inst5, theta5, mom5, lr=LR, momentum=MU, nesterov=True), n=10)
+    time_alone("acc5", acc5_only)
     mean_grad_ms = max(g1.elapsed_time(g2) / reps - gram_only_ms, 1e-6)
     direct_ms = g3.elapsed_time(g4) / reps
     pair_ms = g4.elapsed_time(g5) / reps
@@ -467,6 +493,13 @@ def run_ours(args, rank, world, local_rank):
         "outer_step_kernel_large": hbm_entry(ab["os5"], sec_ms["os5"], ms_per_launch=sec_ms["os5"], section="configs[4] outer step K=4, P=1.3e9"),
         "norm_test_kernel_micro": hbm_entry(ab["acc5"], sec_ms["acc5"], ms_per_launch=sec_ms["acc5"] / C5_MICRO,
                                             section="configs[4] accumulate x8 + finalize (incl. the reset of S)"),
+        "streaming_kernels_alone": {
+            "note": "the same four kernels timed by themselves after a 1 s pause (20 launches each, clocks unconstrained)",
+            "norm_test_kernel": hbm_entry(ab["nt2"], alone["nt2"]),
+            "outer_step_kernel": hbm_entry(ab["os2"], alone["os2"]),
+            "outer_step_kernel_large": hbm_entry(ab["os5"], alone["os5"]),
+            "norm_test_kernel_micro": hbm_entry(ab["acc5"], alone["acc5"], includes="the 8 accumulate launches, no reset / finalize"),
+        },
         "gram_path": tensor_entry(sym + mg, sec_ms["gram3"], tpeak, ms_per_step=sec_ms["gram3"],
                                   executed_tflops=(executed + mg) / (sec_ms["gram3"] * 1e-3) / 1e12, peak_regime=regime,
                                   includes="configs[2]: reset + gram + mean-grad + accumulate + finalize, inside the step"),

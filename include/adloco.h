@@ -112,8 +112,9 @@ typedef struct {
 
 /* ---- context ------------------------------------------------------------ */
 
-/* Creates a context on CUDA device `device` (allocates a few MB of workspace;
- * synchronous).  *out is NULL on failure. */
+/* Creates a context on CUDA device `device` (allocates about 10 MB of workspace, sized
+ * for the largest batch the streaming entry points take, so that none of them allocates
+ * or synchronises later; synchronous).  *out is NULL on failure. */
 int adloco_create(adloco_ctx** out, int device);
 /* Frees the workspace.  The caller must have synchronised every stream that used it. */
 int adloco_destroy(adloco_ctx* ctx);
@@ -370,7 +371,8 @@ int adloco_accum_finalize(adloco_ctx* ctx, adloco_accum* acc, const adloco_test_
  *   inst_writeback  HOST array of K dev pointers (may be NULL, entries may be NULL):
  *                each receives theta' rounded to inst_dtype (Algorithm 3 resets every
  *                worker to the trainer's parameters at the next outer step)
- * fp32 arithmetic, the K differences summed in the order k = 0..K-1. */
+ * The K differences (each exact in fp64) are summed in fp64 in the order k = 0..K-1 and the
+ * update is carried in fp64; every output element is rounded to fp32 once. */
 int adloco_outer_step(adloco_ctx* ctx, const void* const* inst_params, adloco_dtype inst_dtype, int32_t K,
                       int64_t P, const float* theta_in, float* theta_out, const float* mom_in, float* mom_out,
                       float lr, float momentum, int nesterov, void* const* inst_writeback, void* stream);

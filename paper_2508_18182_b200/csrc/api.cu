@@ -89,6 +89,9 @@ int adloco_create(adloco_ctx** out, int device) {
     ctx->max_grid = ctx->sm_count * 8;
     bool ok = true;
     ok = ok && cudaMalloc(&ctx->blk_scalars, (size_t)ctx->max_grid * 4 * sizeof(double)) == cudaSuccess;
+    // per-block partial row sums for the largest launch: at most 4 resident blocks per SM, kMaxBatchRows rows
+    ctx->n_partials_elems = (size_t)ctx->sm_count * 4 * (size_t)kMaxBatchRows;
+    ok = ok && cudaMalloc(&ctx->n_partials, ctx->n_partials_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->ticket, 64) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->scratch_sums, sizeof(adloco_test_sums)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->gemm_status, 64) == cudaSuccess;

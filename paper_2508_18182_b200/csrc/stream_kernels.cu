@@ -379,6 +379,8 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
     }
 }
 
+// The workspace is sized at creation for the largest launch, so this never allocates in
+// practice; it stays as the guard for a device with more resident blocks per SM than assumed.
 static int grow_workspace(adloco_ctx* ctx, size_t need_elems) {
     if (need_elems <= ctx->n_partials_elems) return ADLOCO_OK;
     if (ctx->n_partials) {
