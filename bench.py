@@ -101,9 +101,14 @@ def aggregate_throughput(units_per_rank: float, world: int, max_seconds: float) 
 
 
 # DRAM traffic of norm_test_kernel per gradient element, from the ncu capture of the
-# profiling case (B=64, P=2^21: 536.98 MB read + 4.10 MB written for 2^27 elements);
+# profiling case (B=64, P=2^21: 537.0 MB read + 1.63 MB written for 2^27 elements);
 # traffic grows in proportion to B*P, so a full launch is this times its element count.
-NT_TRAFFIC_BYTES_PER_ELEMENT = (536.98e6 + 4.10e6) / float(64 * (1 << 21))
+NT_TRAFFIC_BYTES_PER_ELEMENT = (537.0e6 + 1.63e6) / float(64 * (1 << 21))
+# DRAM traffic of the grouped direct kernel (CTA-pair form) per transformer block of four
+# layers at B=32, T=1024, from the ncu capture of the profiling case (one block: 902.3 MB
+# read + 24.0 MB written for 805.3 MB of operands); every block's operands are read once,
+# so a launch over n blocks moves n times this.
+DG_TRAFFIC_BYTES_PER_BLOCK = 902.34e6 + 24.0e6
 
 
 def load_peaks():
@@ -486,6 +491,7 @@ def run_ours(args, rank, world, local_rank):
         return d
 
     model_ms = sec_ms["model4"]
+    kernel_is_pair = True     # the automatic route takes the CTA-pair kernel on every device that launches clusters
     kernels = {
         "norm_test_kernel": hbm_entry(ab["nt2"], sec_ms["nt2"], ms_per_launch=sec_ms["nt2"], section="configs[1] norm test + eta sweep",
                                       traffic=NT_TRAFFIC_BYTES_PER_ELEMENT * NT_B * NT_P),
@@ -520,7 +526,9 @@ def run_ours(args, rank, world, local_rank):
     # the dominant kernel of the step by time: the direct per-sample-gradient GEMM of the whole model
     roofline = tensor_entry(mflops / mlaunches, model_ms / mlaunches, tpeak, kernel="direct_group_kernel",
                             ms_per_launch=model_ms / mlaunches, launches_per_step=mlaunches, peak_regime=regime,
-                            peak_source=peaks["source"], traffic=None,
+                            peak_source=peaks["source"],
+                            traffic=(DG_TRAFFIC_BYTES_PER_BLOCK * len(C4_SHAPES) / 4 if kernel_is_pair else None),
+                            operand_bytes=sum(2 * C4_B * GR_T * (di + do) for di, do in C4_SHAPES),
                             section="configs[3]: one launch per micro-batch over its 48 layers (adloco_linear_sqnorm_group, "
                                     "automatic route); flops per launch = sum over the layers of 2 b T d_in d_out")
     line = {
@@ -659,6 +667,7 @@ def run_table(args):
     ms_g = gpu_ms(lambda: ctx.gram_sqnorm(X, D, n))
     ms_gs = gpu_ms(lambda: ctx.gram_sqnorm(X, D, n, grad_sum=S))
     ms_d = gpu_ms(lambda: ctx.linear_sqnorm(X, D, n, grad_sum=S, method="direct"))
+    ms_p = gpu_ms(lambda: ctx.linear_sqnorm(X, D, n, grad_sum=S, method="pair"))
     Xn, Dn = W.to_numpy(X), W.to_numpy(D)
     o_s = cpu_s(lambda: O.linear_layer_terms(Xn, Dn))
     emit(3, "gram_sqnorm (norms only)", ms_g, flops=sym, note=f"executed {executed / (ms_g * 1e-3) / 1e12:.0f} TFLOP/s")
@@ -666,6 +675,7 @@ def run_table(args):
     emit(3, "mean-gradient GEMM (difference)", ms_gs - ms_g, flops=mg)
     emit(3, "linear_sqnorm direct (norms + gradient sum)", ms_d, flops=mg, oracle_s=o_s, oracle_note="whole",
          note="same outputs as the row above from one GEMM")
+    emit(3, "linear_sqnorm pair (CTA-pair direct kernel)", ms_p, flops=mg, oracle_s=o_s, oracle_note="whole")
     Sb = torch.zeros(GR_DOUT, device=dev)
     ms_b = gpu_ms(lambda: ctx.vector_param_sqnorm(D, n, grad_sum=Sb), flush=True)
     Dn8 = Dn[:8]
@@ -709,48 +719,25 @@ def run_table(args):
     o4 = cpu_s(lambda: [O.linear_layer_terms(x, d) for x, d in Xb]) * 48
     emit(4, "whole model, Gram route (48 layers x 4 micro-batches + finalize)", ms4, flops=f_sym + f_mg, oracle_s=o4,
          oracle_note="one block x one micro-batch timed, x48 extrapolated")
-    ms4d = gpu_ms(lambda: whole_model("auto"), reps=5, warm=1)
-    emit(4, "whole model, linear_sqnorm auto (direct route)", ms4d, flops=f_mg, oracle_s=o4, oracle_note="as above")
-    # the layers of a micro-batch are independent (they only add into n and into their own S): issued
-    # alternately on two streams, the tail of one layer's kernel overlaps the head of the next
-    s_a, s_b = torch.cuda.Stream(), torch.cuda.Stream()
+    ms4d = gpu_ms(lambda: whole_model("direct"), reps=5, warm=1)
+    emit(4, "whole model, one-CTA direct kernel, one launch per layer", ms4d, flops=f_mg, oracle_s=o4, oracle_note="as above")
+    ms4p = gpu_ms(lambda: whole_model("auto"), reps=5, warm=1)
+    emit(4, "whole model, linear_sqnorm auto (CTA-pair direct kernel), one launch per layer", ms4p, flops=f_mg, oracle_s=o4,
+         oracle_note="as above")
+    groups = [ctx.make_layer_group([(Xl, Dl, S) for (Xl, Dl), S in zip(data[j], sums)]) for j in range(4)]
 
-    def whole_model_two_streams():
-        main = torch.cuda.current_stream()
+    def whole_model_grouped(method):
         acc.reset()
         for j in range(4):
-            n_mb.zero_()                                   # every layer adds into n with atomics
-            s_a.wait_stream(main)
-            s_b.wait_stream(main)
-            for l, (Xl, Dl) in enumerate(data[j]):
-                ctx.linear_sqnorm(Xl, Dl, n_mb, accumulate_norms=True, grad_sum=sums[l], accumulate_sum=True,
-                                  method="auto", stream=(s_a if (l & 1) == 0 else s_b))
-            main.wait_stream(s_a)
-            main.wait_stream(s_b)
+            ctx.linear_sqnorm_group(groups[j], n_mb, method=method, accumulate_sum=True)
             acc.accumulate(per_sample_sqnorm=n_mb)
         acc.finalize(p4, sync=False)
-    try:
-        ms4s = gpu_ms(whole_model_two_streams, reps=5, warm=1)
-        emit(4, "whole model, direct route, layers alternating on two streams", ms4s, flops=f_mg, oracle_s=o4,
-             oracle_note="as above")
-    except Exception as exc:
-        print(json.dumps({"config": 4, "kernel": "two streams", "skipped": str(exc)[:200]}), flush=True)
-    # the same 192 calls captured once into a CUDA graph and replayed (nothing in them synchronises)
-    try:
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            whole_model("auto")
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            whole_model("auto")
-        ms4g = gpu_ms(graph.replay, reps=5, warm=1)
-        emit(4, "whole model, direct route, replayed as one CUDA graph", ms4g, flops=f_mg, oracle_s=o4, oracle_note="as above")
-        del graph
-    except Exception as exc:   # capture is an extra, not part of the path
-        print(json.dumps({"config": 4, "kernel": "CUDA graph replay", "skipped": str(exc)[:200]}), flush=True)
+    ms4g1 = gpu_ms(lambda: whole_model_grouped("direct"), reps=5, warm=1)
+    emit(4, "whole model, linear_sqnorm_group (one-CTA kernel), one launch per micro-batch", ms4g1, flops=f_mg, oracle_s=o4,
+         oracle_note="as above")
+    ms4g2 = gpu_ms(lambda: whole_model_grouped("auto"), reps=5, warm=1)
+    emit(4, "whole model, linear_sqnorm_group auto (CTA-pair kernel), one launch per micro-batch", ms4g2, flops=f_mg,
+         oracle_s=o4, oracle_note="as above")
     acc.close()
     del data, sums
     torch.cuda.empty_cache()
