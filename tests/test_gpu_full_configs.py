@@ -109,15 +109,17 @@ def test_config3_gram_layer_full_size(ctx):
 
 # ---------------------------------------------------------------- config 4
 def test_config4_whole_model_switch_mode_full_size(ctx):
-    """12 blocks x 4 linear layers, batch 128 as 4 accumulated micro-batches of 32, by both routes
-    (the Gram identity, and whatever route AUTO picks: the direct one for these shapes).  The oracle
+    """12 blocks x 4 linear layers, batch 128 as 4 accumulated micro-batches of 32, three ways: the
+    Gram identity layer by layer, the automatic route layer by layer (the direct kernel over CTA pairs
+    for these shapes), and the grouped call that takes the 48 layers of a micro-batch in ONE launch --
+    the launch configuration the benchmark times.  The oracle
     runs the whole model once, streamed layer by layer and micro-batch by micro-batch (explicit
     per-sample gradients in fp64; about a minute of host BLAS), and every output is compared: the
     128 per-sample norms, each layer's gradient sum element by element, ||S_l||^2 per layer, and the
     statistic, decision and switch plan."""
     shapes = list(W.GPT2_SMALL_BLOCK_LINEARS) * 12
     n_micro, b, T = 4, 32, 1024
-    routes = ("gram", "auto")
+    routes = ("gram", "auto", "group")
     sums = {m: [torch.empty(do, di, device=DEV) for di, do in shapes] for m in routes}
     accs = {m: A.Accumulator(ctx, sums[m]) for m in routes}
     n_mb = {m: torch.zeros(b, device=DEV) for m in routes}
@@ -127,15 +129,18 @@ def test_config4_whole_model_switch_mode_full_size(ctx):
     n_ref = np.zeros(n_micro * b)
     S_ref = [np.zeros((do, di)) for di, do in shapes]
     for j in range(n_micro):
-        for l, (di, do) in enumerate(shapes):
-            X, D = W.linear_layer(b, T, di, do, seed=100000 + 100 * l + j, device=DEV)
-            for m in routes:
+        # the grouped launch needs every layer of the micro-batch resident at once (9.7 GB)
+        data = [W.linear_layer(b, T, di, do, seed=100000 + 100 * l + j, device=DEV) for l, (di, do) in enumerate(shapes)]
+        ctx.linear_sqnorm_group([(X, D, S) for (X, D), S in zip(data, sums["group"])], n_mb["group"], method="auto",
+                                accumulate_sum=True)
+        for l, (X, D) in enumerate(data):
+            for m in ("gram", "auto"):
                 ctx.linear_sqnorm(X, D, n_mb[m], accumulate_norms=(l > 0), grad_sum=sums[m][l], accumulate_sum=True,
                                   method=m)
             n_l, S_l = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))     # overlaps the GPU work
             n_ref[j * b:(j + 1) * b] += n_l
             S_ref[l] += S_l
-            del X, D
+        del data
         for m in routes:
             accs[m].accumulate(per_sample_sqnorm=n_mb[m])
             n_all[m][j * b:(j + 1) * b] = n_mb[m]
