@@ -382,7 +382,7 @@ def run_ours(args, rank, world, local_rank):
     # the tensor-core kernels of one layer one by one (outside the timed steps): the call without a
     # sum buffer runs the Gram kernel alone, the difference to the full call is the GEMM
     reps = 20
-    g0, g1, g2, g3, g4, g5 = ev(), ev(), ev(), ev(), ev(), ev()
+    g0, g1, g2, g3, g4, g5, g6 = ev(), ev(), ev(), ev(), ev(), ev(), ev()
     torch.cuda.synchronize()
     time.sleep(1.0)           # let the clocks recover from the timed region: these are burst figures
     g0.record(stream)
@@ -400,8 +400,12 @@ def run_ours(args, rank, world, local_rank):
     for _ in range(reps):
         ctx.linear_sqnorm(X, D, n_layer, grad_sum=S_layer, accumulate_sum=True, method="pair")
     g5.record(stream)
+    for _ in range(reps):
+        ctx.linear_sqnorm(X, D, n_layer, method="gram_pair")
+    g6.record(stream)
     torch.cuda.synchronize()
     gram_only_ms = g0.elapsed_time(g1) / reps
+    gram_pair_ms = g5.elapsed_time(g6) / reps
     # the streaming kernels by themselves, after a pause that lets the clocks recover from the power cap
     # the tensor-core sections of the step run into (the cap holds the SM clock, and with it the on-chip
     # network, well below its maximum for the whole step)
@@ -437,6 +441,8 @@ def run_ours(args, rank, world, local_rank):
     stream_ms = sec_ms["nt2"] + sec_ms["os2"] + sec_ms["os5"] + sec_ms["acc5"]
     value = aggregate_throughput(stream_bytes, world, stream_ms * 1e-3) / 1e9
     sym, executed, mg = gram_flops()
+    m256 = (GR_T + 255) // 256
+    executed_pair = 2 * GR_B * (m256 * (m256 + 1) // 2) * 256 * 256 * (GR_DIN + GR_DOUT)
     mflops, mlaunches = model_flops()
 
     # ---- end to end through the host-memory entry points (rank-local pinned buffers): the
@@ -514,6 +520,11 @@ def run_ours(args, rank, world, local_rank):
         "gram_sqnorm_kernel": tensor_entry(sym, gram_only_ms, burst, ms_per_launch=gram_only_ms,
                                            executed_tflops=executed / (gram_only_ms * 1e-3) / 1e12,
                                            timed="alone, 20 launches back to back (a burst), incl. the memset of n"),
+        "gram_pair_kernel": tensor_entry(sym, gram_pair_ms, burst, ms_per_launch=gram_pair_ms,
+                                         executed_tflops=executed_pair / (gram_pair_ms * 1e-3) / 1e12,
+                                         timed="alone, 20 launches back to back: the Gram identity over CTA pairs "
+                                               "(256-token blocks; the sub-block below the diagonal of a diagonal "
+                                               "block is computed and dropped)"),
         "mean_grad_kernel": tensor_entry(mg, mean_grad_ms, burst, ms_per_launch=mean_grad_ms,
                                          timed="alone: full call minus the Gram-only call"),
         "direct_sqnorm_kernel_one_layer": tensor_entry(mg, direct_ms, burst, ms_per_launch=direct_ms,

@@ -266,7 +266,8 @@ int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
  *   ADLOCO_LINEAR_AUTO    whichever executes fewer tensor-core flops for the shape
  *                         (direct wins when T exceeds about d_in d_out / (d_in + d_out));
  *                         the direct route then runs in its pair form where available. */
-enum { ADLOCO_LINEAR_AUTO = 0, ADLOCO_LINEAR_GRAM = 1, ADLOCO_LINEAR_DIRECT = 2, ADLOCO_LINEAR_DIRECT_PAIR = 3 };
+enum { ADLOCO_LINEAR_AUTO = 0, ADLOCO_LINEAR_GRAM = 1, ADLOCO_LINEAR_DIRECT = 2, ADLOCO_LINEAR_DIRECT_PAIR = 3,
+       ADLOCO_LINEAR_GRAM_ONE_CTA = 4, ADLOCO_LINEAR_GRAM_PAIR = 5 };
 int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                          int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
                          int accumulate_sum, int method, void* stream);

@@ -69,7 +69,7 @@ class LinearLayer(C.Structure):
                 ("grad_sum", C.c_void_p)]
 
 
-LINEAR_METHODS = {"auto": 0, "gram": 1, "direct": 2, "pair": 3}
+LINEAR_METHODS = {"auto": 0, "gram": 1, "direct": 2, "pair": 3, "gram_one_cta": 4, "gram_pair": 5}
 
 
 class AdlocoError(RuntimeError):

@@ -282,9 +282,10 @@ int adloco_inner_product_test(adloco_ctx* ctx, const void* grads, adloco_dtype d
 // ---------------------------------------------------------------------------------
 // Gram path
 // ---------------------------------------------------------------------------------
-int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
-                       int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
-                       int accumulate_sum, void* stream) {
+// variant: 0 = the one-CTA Gram kernel, 1 = the CTA-pair Gram kernel, -1 = whichever suits the shape
+static int gram_route(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                      int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
+                      int accumulate_sum, int variant, void* stream) {
     if (!ctx || !X || !D || !per_sample_sqnorm) return ADLOCO_ERR_INVALID_ARG;
     if (B < 1 || T < 1 || d_in < 1 || d_out < 1) return ADLOCO_ERR_INVALID_ARG;
     if ((d_in % 8) != 0 || (d_out % 8) != 0) return ADLOCO_ERR_UNSUPPORTED;
@@ -293,10 +294,20 @@ int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     if (grad_sum && !aligned16(grad_sum)) return ADLOCO_ERR_ALIGNMENT;
     DeviceGuard g(ctx->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int rc = launch_gram_sqnorm(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, st);
+    if (variant == 1 && !pair_launch_ok(ctx)) return ADLOCO_ERR_UNSUPPORTED;
+    if (variant < 0) variant = 0;
+    int rc = variant == 1 ? launch_gram_pair(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, 1, st)
+                          : launch_gram_sqnorm(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, st);
     if (rc != ADLOCO_OK) return rc;
     if (grad_sum) rc = launch_mean_grad(ctx, X, D, B, T, d_in, d_out, grad_sum, accumulate_sum, st);
     return rc;
+}
+
+int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                       int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
+                       int accumulate_sum, void* stream) {
+    return gram_route(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, grad_sum, accumulate_sum, -1,
+                      stream);
 }
 
 int adloco_vector_param_sqnorm(adloco_ctx* ctx, const void* D, const void* X, int64_t B, int64_t T, int64_t d,
@@ -328,10 +339,13 @@ int adloco_linear_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t 
                          int64_t d_out, float* per_sample_sqnorm, int accumulate_norms, float* grad_sum,
                          int accumulate_sum, int method, void* stream) {
     if (method != ADLOCO_LINEAR_AUTO && method != ADLOCO_LINEAR_GRAM && method != ADLOCO_LINEAR_DIRECT &&
-        method != ADLOCO_LINEAR_DIRECT_PAIR)
+        method != ADLOCO_LINEAR_DIRECT_PAIR && method != ADLOCO_LINEAR_GRAM_ONE_CTA && method != ADLOCO_LINEAR_GRAM_PAIR)
         return ADLOCO_ERR_INVALID_ARG;
     if (!ctx || !X || !D || !per_sample_sqnorm) return ADLOCO_ERR_INVALID_ARG;
     if (B < 1 || T < 1 || d_in < 1 || d_out < 1) return ADLOCO_ERR_INVALID_ARG;
+    if (method == ADLOCO_LINEAR_GRAM_ONE_CTA || method == ADLOCO_LINEAR_GRAM_PAIR)
+        return gram_route(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, grad_sum, accumulate_sum,
+                          method == ADLOCO_LINEAR_GRAM_PAIR ? 1 : 0, stream);
     const bool was_auto = (method == ADLOCO_LINEAR_AUTO);
     if (method == ADLOCO_LINEAR_AUTO) {
         // tensor work of the two routes at the granularity the kernels execute, divided by

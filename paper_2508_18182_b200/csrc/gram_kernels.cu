@@ -27,6 +27,7 @@ using namespace ptx;
 
 constexpr int kDirectGroupCap = 48;                 // layers per launch of the grouped direct kernel
 constexpr uint64_t kDrainLimitNs = 50000000ull;    // 50 ms per barrier while leaving after a time-out
+constexpr uint64_t kPairGraceNs = 1000000ull;      // 1 ms: a CTA pair leaving after a time-out; copies in flight land long before
 
 struct PipeState {
     uint32_t stage = 0, phase = 0;
@@ -249,6 +250,283 @@ gram_sqnorm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
+}
+
+// =====================================================================================
+// Gram kernel over CTA pairs
+// =====================================================================================
+// The T x T Gram matrices are cut into 256-token blocks; a work item is (sample i, block
+// row p, block column q >= p).  The two CTAs of a cluster share one 256 x 256 MMA per K
+// step (cta_group::2): CTA r holds token rows 256 p + 128 r .. + 127 in its tensor memory
+// and loads those rows (16 KB per stage) plus ONE half of the column operand, tokens
+// 256 q + 128 r .. + 127 (16 KB) -- 32 KB per stage per CTA for a 128 x 256 tile of
+// output, 131 flops per byte brought into shared memory against 87 for the one-CTA item
+// (whose feed of operands, not the tensor pipe, sets its time).  On the diagonal (p == q)
+// a CTA's row tile IS its column half and is fetched once.  Of a diagonal item's four
+// 128 x 128 sub-blocks the one below the diagonal is computed and not used (weight 0);
+// blocks beyond T read as zeros.
+//
+// The X X^T product (TMEM columns 0-255) is complete before the D D^T product (columns
+// 256-511) starts: the 16 epilogue warps copy their 64 columns of X X^T into registers
+// while the D D^T MMAs run and hand the columns back, so the next item's X X^T MMAs start
+// the moment this item's D D^T MMAs have been issued and the tensor pipe never waits for
+// the epilogue; the elementwise product is then formed against D D^T straight from TMEM.
+//
+// Items are drawn in list order (sample-major) from a global counter, so all workers sit
+// on the same few samples at a time and those samples' operands stay in L2.
+constexpr int GP_STAGES = 7;                                   // 224 KB of operands in flight: 7 stages measured 5 % faster than 6, 6 % than 4
+constexpr int GP_STAGE_BYTES = 2 * GR_BLOCK_BYTES;             // row tile + this CTA's half of the columns: 32 KB
+constexpr int GP_EPI_WARPS = 16;                               // four column slices of 64 per TMEM lane quarter
+constexpr int GP_THREADS = 64 + 32 * GP_EPI_WARPS;             // warp 0 TMA, warp 1 MMA, the rest epilogue
+constexpr int GP_SCHED_Q = 8;
+constexpr int GP_SMEM = GP_STAGES * GP_STAGE_BYTES + 1024 /*align*/ + 512 /*barriers*/;
+
+struct GramPairArgs {
+    int B, T, d_in, d_out;
+    int nt;               // 128-token blocks per side
+    int m;                // 256-token blocks per side
+    int rects;            // items per sample: m (m + 1) / 2, or m (m - 1) / 2 when the diagonal is left out
+    int with_diag;        // 0: only items with q > p
+    int total_items;
+    int* counter;         // zero at launch
+    float* n;             // [B], +=
+    int* status;
+    uint64_t wait_ns;
+};
+
+__device__ __forceinline__ void gram_pair_decode(int item, const GramPairArgs& a, int& i, int& p, int& q) {
+    i = item / a.rects;
+    int r = item - i * a.rects;
+    const int first = a.with_diag ? 0 : 1;        // offset of the first block column of a row from its diagonal
+    for (p = 0; p < a.m - 1; ++p) {
+        const int cnt = a.m - p - first;
+        if (r < cnt) break;
+        r -= cnt;
+    }
+    q = p + first + r;
+}
+
+__global__ void __launch_bounds__(GP_THREADS, 1)
+gram_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
+                 const GramPairArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_base = smem_base + GP_STAGES * GP_STAGE_BYTES;
+    auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (GP_STAGES + s); };
+    const uint32_t xx_full = bar_base + 8u * (2 * GP_STAGES);
+    const uint32_t dd_full = bar_base + 8u * (2 * GP_STAGES + 1);
+    const uint32_t xx_empty = bar_base + 8u * (2 * GP_STAGES + 2);
+    const uint32_t dd_empty = bar_base + 8u * (2 * GP_STAGES + 3);
+    const uint32_t drain_bar = bar_base + 8u * (2 * GP_STAGES + 4);
+    auto sched_full = [&](uint32_t s) { return bar_base + 8u * (2 * GP_STAGES + 5 + s); };
+    auto sched_empty = [&](uint32_t s) { return bar_base + 8u * (2 * GP_STAGES + 5 + GP_SCHED_Q + s); };
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ int sched_item[GP_SCHED_Q];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();          // 0 = the CTA that issues the MMAs and draws the items
+    const int worker = (int)(blockIdx.x >> 1);
+    const int n_workers = (int)(gridDim.x >> 1);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (uint32_t s = 0; s < (uint32_t)GP_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(xx_full, 1);
+        mbar_init(dd_full, 1);
+        mbar_init(xx_empty, 2 * GP_EPI_WARPS);          // the epilogue warps of both CTAs
+        mbar_init(dd_empty, 2 * GP_EPI_WARPS);
+        mbar_init(drain_bar, 1);
+        for (uint32_t s = 0; s < (uint32_t)GP_SCHED_Q; ++s) {
+            mbar_init(sched_full(s), 1);
+            // readers of a slot: the even CTA's MMA thread, the odd CTA's TMA thread, both CTAs' epilogue warps
+            mbar_init(sched_empty(s), 2 * (1 + GP_EPI_WARPS));
+        }
+        fence_barrier_init();
+        prefetch_tmap(&tmX);
+        prefetch_tmap(&tmD);
+    }
+    if (warp == 1) { tmem_alloc_pair(smem_u32(&tmem_base_slot), 512); tmem_relinquish_pair(); }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();        // the peer's barriers exist before anything is signalled on them
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+    const int kx = (a.d_in + GR_BK - 1) / GR_BK, kd = (a.d_out + GR_BK - 1) / GR_BK;
+    const int chunks = kx + kd;
+    const uint32_t sched_empty_remote0 = map_to_cta(sched_empty(0), 0);
+
+    // item number k of this worker, as published by the drawing thread; -1 when the wait ran out
+    auto take_item = [&](int k, bool whole_warp) -> int {
+        const uint32_t slot = (uint32_t)k % GP_SCHED_Q, ph = ((uint32_t)k / GP_SCHED_Q) & 1u;
+        bool got = mbar_wait<true>(sched_full(slot), ph, abortp, a.wait_ns);
+        if (whole_warp) got = __all_sync(0xffffffffu, got);
+        if (!got) return -1;
+        const int item = *reinterpret_cast<volatile int*>(&sched_item[slot]);
+        if (whole_warp) __syncwarp();
+        if (!whole_warp || lane == 0) {
+            if (rank != 0) mbar_arrive_cluster(sched_empty_remote0 + 8u * slot);
+            else mbar_arrive(sched_empty(slot));
+        }
+        return item;
+    };
+
+    if (warp == 0) {
+        // ---------------- TMA producer (one per CTA; the even CTA's also draws the items) ----------------
+        if (lane == 0) {
+            PipeState ps;
+            bool ok = true;
+            int item = worker;                      // the first item needs no draw
+            for (int k = 0; ok; ++k) {
+                if (rank == 0) {
+                    const uint32_t slot = (uint32_t)k % GP_SCHED_Q, ph = ((uint32_t)k / GP_SCHED_Q) & 1u;
+                    if (!mbar_wait<true>(sched_empty(slot), ph ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
+                    *reinterpret_cast<volatile int*>(&sched_item[slot]) = item;
+                    st_cluster_u32(map_to_cta(smem_u32(&sched_item[slot]), 1u), (uint32_t)item);
+                    mbar_arrive(sched_full(slot));
+                    mbar_arrive_cluster(map_to_cta(sched_full(slot), 1u));
+                } else {
+                    item = take_item(k, false);
+                    if (item < 0) { ok = false; break; }
+                }
+                if (item >= a.total_items) break;   // the list is exhausted: every role has been told
+                int next_item = 0;
+                if (rank == 0) next_item = n_workers + atomicAdd(a.counter, 1);
+                int i, p, q;
+                gram_pair_decode(item, a, i, p, q);
+                const int row0 = (2 * p + (int)rank) * GR_TILE;      // this CTA's token rows
+                const int col0 = (2 * q + (int)rank) * GR_TILE;      // this CTA's half of the token columns
+                const bool diag = (p == q);
+                const uint32_t bytes = diag ? GR_BLOCK_BYTES : GP_STAGE_BYTES;
+                for (int c = 0; c < chunks; ++c) {
+                    if (!mbar_wait(empty_bar(ps.stage), ps.phase ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
+                    const bool is_x = c < kx;
+                    const CUtensorMap* map = is_x ? &tmX : &tmD;
+                    const int k0 = (is_x ? c : c - kx) * GR_BK;
+                    const uint32_t sA = smem_base + ps.stage * GP_STAGE_BYTES;
+                    const uint32_t bar = map_to_cta(full_bar(ps.stage), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(full_bar(ps.stage), 2 * bytes);
+                    tma_load_3d_pair(sA, map, bar, k0, row0, i);
+                    if (!diag) tma_load_3d_pair(sA + GR_BLOCK_BYTES, map, bar, k0, col0, i);
+                    ps.advance(GP_STAGES);
+                }
+                item = next_item;
+            }
+            if (!ok) {
+                // leaving after a time-out: the byte counts of copies in flight complete on the even CTA's
+                // barriers, which the odd CTA cannot wait on: both sit out a grace period far beyond the
+                // flight time of a copy
+                st_cluster_u32(map_to_cta(smem_u32(&abort_flag), rank ^ 1u), 1u);
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < kPairGraceNs) { }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (even CTA only) ----------------
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(256, 256, 0, 0);     // both operands K-major
+            PipeState ps;
+            bool ok = true;
+            for (int k = 0; ok; ++k) {
+                const int item = take_item(k, false);
+                if (item < 0) { ok = false; break; }
+                if (item >= a.total_items) break;
+                int i, p, q;
+                gram_pair_decode(item, a, i, p, q);
+                const uint32_t b_off = (p == q) ? 0u : (uint32_t)GR_BLOCK_BYTES;   // on the diagonal the row tile is the column half
+                for (int c = 0; c < chunks; ++c) {
+                    if (c == 0 || c == kx) {
+                        // the accumulator about to be overwritten has been read by every epilogue warp
+                        if (!mbar_wait<true>(c == 0 ? xx_empty : dd_empty, ((uint32_t)k & 1u) ^ 1u, abortp, a.wait_ns)) { ok = false; break; }
+                        tc_fence_after();
+                    }
+                    if (!mbar_wait(full_bar(ps.stage), ps.phase, abortp, a.wait_ns)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t acc = tmem_base + (c < kx ? 0u : 256u);
+                    const bool first = (c == 0 || c == kx);
+                    const uint32_t sA = smem_base + ps.stage * GP_STAGE_BYTES;
+                    const uint32_t sB = sA + b_off;
+#pragma unroll
+                    for (int kk = 0; kk < GR_BK / 16; ++kk) {
+                        // K-major, 128-byte swizzle: rows of 128 B, 8-row groups 1024 B apart; 16 features
+                        // further along K = 32 bytes further in the row
+                        const uint64_t da = smem_desc_sw128(sA + kk * 32, 16, 1024);
+                        const uint64_t db = smem_desc_sw128(sB + kk * 32, 16, 1024);
+                        mma_bf16_pair(acc, da, db, idesc, (first && kk == 0) ? 0u : 1u);
+                    }
+                    mma_commit_pair(empty_bar(ps.stage), 3);       // the stage is free in both CTAs
+                    ps.advance(GP_STAGES);
+                    if (c == kx - 1) mma_commit_pair(xx_full, 3);  // X X^T of this item complete in both CTAs
+                }
+                if (ok) mma_commit_pair(dd_full, 3);
+            }
+            if (!ok) {
+                st_cluster_u32(map_to_cta(smem_u32(&abort_flag), 1u), 1u);
+                mma_commit_pair(drain_bar, 1);
+                int never = 0;
+                mbar_wait(drain_bar, 0, &never, kDrainLimitNs);
+            }
+        }
+    } else {
+        // ---------------- epilogue: sum over the tile of (X X^T) .* (D D^T) ----------------
+        const uint32_t lq = warp & 3;                    // TMEM lane quarter: rows 32 lq .. 32 lq + 31 of this CTA's row tile
+        const uint32_t slice = (uint32_t)(warp - 2) >> 2;   // columns 64 slice .. 64 slice + 63 of the 256
+        const uint32_t xx_empty_remote = map_to_cta(xx_empty, 0), dd_empty_remote = map_to_cta(dd_empty, 0);
+        const uint32_t taddr = tmem_base + ((lq * 32u) << 16) + slice * 64u;
+        for (int k = 0;; ++k) {
+            const int item = take_item(k, true);
+            if (item < 0 || item >= a.total_items) break;
+            int i, p, q;
+            gram_pair_decode(item, a, i, p, q);
+            // weight of this warp's 128 x 128 sub-block: 0 below the diagonal or beyond T (never read),
+            // 1 on the diagonal, 2 above it (its mirror image is never computed)
+            const int rb = 2 * p + (int)rank, cb = 2 * q + (int)(slice >> 1);
+            const float w = (rb >= a.nt || cb >= a.nt || rb > cb) ? 0.f : (rb == cb ? 1.f : 2.f);
+            const uint32_t par = (uint32_t)k & 1u;
+            if (!__all_sync(0xffffffffu, mbar_wait(xx_full, par, abortp, a.wait_ns))) break;
+            tc_fence_after();
+            uint32_t xx[4][16];
+            if (w != 0.f) {                              // uniform across the warp
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) tmem_ld16(taddr + cc * 16, xx[cc]);
+                tmem_ld_wait();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(xx_empty_remote);
+            if (!__all_sync(0xffffffffu, mbar_wait(dd_full, par, abortp, a.wait_ns))) break;
+            tc_fence_after();
+            float sum = 0.f;
+            if (w != 0.f) {
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t r[16];
+                    tmem_ld16(taddr + 256u + cc * 16, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) sum = fmaf(__uint_as_float(xx[cc][e]), __uint_as_float(r[e]), sum);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(dd_empty_remote);
+            if (w != 0.f) {
+                const float tot = warp_sum_f(sum) * w;
+                if (lane == 0) atomicAdd(a.n + i, tot);
+            }
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();   // neither CTA frees tensor memory or leaves while its peer still works
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, 512);
     }
     if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
 }
@@ -724,7 +1002,6 @@ constexpr int DR_STAGING = DR_EPI_WARPS * DR_BOX_OUT;
 constexpr int DR_CHUNKS_MAX = 4;
 constexpr int DR_COLS = DR_CHUNKS_MAX * 16;
 constexpr int DR_THREADS = 64 + 32 * DR_EPI_WARPS;  // warp 0 TMA, warp 1 MMA, the rest epilogue
-constexpr uint64_t kPairGraceNs = 1000000ull;       // 1 ms: leaving after a time-out, copies in flight land long before
 constexpr int DR_SCHED_Q = 8;                       // slots of the item queue between the TMA thread and the other roles
 
 template <bool PAIR>
@@ -1221,6 +1498,50 @@ int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     const int grid = a.total_items < ctx->sm_count ? a.total_items : ctx->sm_count;
     gram_sqnorm_kernel<<<grid, GR_THREADS, GR_SMEM, st>>>(tmX, tmD, a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
+// The CTA-pair form of the Gram kernel; with_diag = 0 leaves the 256-token blocks on the diagonal out
+int launch_gram_pair(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
+                     int64_t d_out, float* n, int accumulate_norms, int with_diag, cudaStream_t st) {
+    CUtensorMap tmX, tmD;
+    int rc = cached_map(ctx, &tmX, X, B, T, d_in, GR_TILE);
+    if (rc != ADLOCO_OK) return rc;
+    rc = cached_map(ctx, &tmD, D, B, T, d_out, GR_TILE);
+    if (rc != ADLOCO_OK) return rc;
+    GramPairArgs a;
+    a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
+    a.nt = (int)((T + GR_TILE - 1) / GR_TILE);
+    a.m = (a.nt + 1) / 2;
+    const int64_t rects = with_diag ? (int64_t)a.m * (a.m + 1) / 2 : (int64_t)a.m * (a.m - 1) / 2;
+    if (rects * B > 0x3fffffff) return ADLOCO_ERR_UNSUPPORTED;
+    a.rects = (int)rects;
+    a.with_diag = with_diag;
+    a.total_items = (int)(rects * B);
+    a.n = n; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
+    if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
+    if (a.total_items == 0) return ADLOCO_OK;
+    a.counter = ctx->sched_counters + (ctx->sched_next.fetch_add(1) % kSchedCounters);
+    ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(a.counter, 0, sizeof(int), st));
+    static std::atomic<bool> attr_set[64];   // the attribute is per device
+    if (!attr_set[ctx->device & 63].load()) {
+        ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(gram_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GP_SMEM));
+        attr_set[ctx->device & 63].store(true);
+    }
+    const int workers = ctx->sm_count / 2;
+    const int grid_workers = a.total_items < workers ? a.total_items : workers;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * grid_workers));
+    cfg.blockDim = dim3(GP_THREADS);
+    cfg.dynamicSmemBytes = GP_SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ADLOCO_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, gram_pair_kernel, tmX, tmD, a));
     ctx->launches++;
     return ADLOCO_OK;
 }

@@ -35,7 +35,7 @@ def _gpu_layer(ctx, X, D, want_S=True, method="gram"):
     return n, S
 
 
-METHODS = ["gram", "direct", "pair", "auto"]
+METHODS = ["gram", "gram_pair", "direct", "pair", "auto"]
 
 
 @pytest.mark.parametrize("method", METHODS)
@@ -140,7 +140,7 @@ def test_whole_model_switch_mode_small(ctx):
     acc.close()
 
 
-@pytest.mark.parametrize("method", METHODS[:3])
+@pytest.mark.parametrize("method", ["gram", "gram_pair", "direct", "pair"])
 def test_a_wait_that_runs_out_raises_the_status_and_the_context_stays_usable(method):
     """Every in-kernel wait is bounded.  With the bound set to one nanosecond the
     first wait that is not satisfied at once gives up: the kernel must leave through

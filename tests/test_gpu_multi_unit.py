@@ -56,13 +56,13 @@ MULTI_UNIT_SHAPES = [
 
 
 @pytest.mark.parametrize("B,T,d_in,d_out", MULTI_UNIT_SHAPES)
-@pytest.mark.parametrize("method", ["direct", "pair", "gram"])
+@pytest.mark.parametrize("method", ["direct", "pair", "gram", "gram_pair"])
 def test_ctas_with_several_units_match_the_oracle(ctx, B, T, d_in, d_out, method):
     X, D = W.linear_layer(B, T, d_in, d_out, seed=7 * B + T, device=DEV)
     _check_layer(ctx, X, D, method, f"{method} B={B} T={T} {d_in}->{d_out}")
 
 
-@pytest.mark.parametrize("method", ["direct", "pair", "gram"])
+@pytest.mark.parametrize("method", ["direct", "pair", "gram", "gram_pair"])
 def test_several_units_exact_on_integers(ctx, method):
     # T = 16 keeps every entry of a per-sample gradient below 2^8 and every sum below 2^24: exact in fp32
     X, D = W.small_integer_layer(11, 16, 768, 1536, seed=5, device=DEV)
@@ -81,6 +81,8 @@ def test_config3_layer_direct_route_full_size(ctx):
     _check_layer(ctx, X, D, "direct", "config 3 direct")
     _check_layer(ctx, X, D, "pair", "config 3 pair")
     _check_layer(ctx, X, D, "auto", "config 3 auto")
+    # the Gram identity over CTA pairs: 320 items of 256 x 256 tokens over 74 pairs, four or five per pair
+    _check_layer(ctx, X, D, "gram_pair", "config 3 Gram over CTA pairs")
 
 
 def test_embedding_with_several_items_per_cta(ctx):
