@@ -16,10 +16,7 @@ namespace adloco {
 
 constexpr int NT_THREADS = 256;
 constexpr int NT_WARPS = NT_THREADS / 32;
-#ifndef ADLOCO_NT_CHUNK
-#define ADLOCO_NT_CHUNK 8
-#endif
-constexpr int NT_CHUNK = ADLOCO_NT_CHUNK;  // rows loaded back to back before they are consumed
+constexpr int NT_CHUNK = 8;  // rows loaded back to back before they are consumed (4 and 16 measured slower)
 
 // ---------------------------------------------------------------------------------
 // small device helpers
@@ -195,6 +192,39 @@ __global__ void decide_kernel(const adloco_test_sums* sums, adloco_test_params p
     if (threadIdx.x == 0 && blockIdx.x == 0) decide_device(*sums, p, out);
 }
 
+// Last block of a reduction: the total over all blocks of the per-block partial sums of 32
+// rows, rows i0 .. i0 + 31.  Warp w adds up blocks w, w + 8, ... for row i0 + lane -- its loads
+// are independent and in flight together, where one thread walking all blocks of a row took
+// a tenth of a 100 us launch -- and the eight warp sums are added in warp order: the order is
+// fixed, so the result is the same on every run.  Called by all threads of the block;
+// returns the total of row i0 + lane in warp 0 (garbage elsewhere and for rows >= B).
+__device__ __forceinline__ double combine_rows32(const float* partials, int64_t B, unsigned nblk, int64_t i0,
+                                                 double (&comb)[NT_WARPS][32]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t i = i0 + lane;
+    double t = 0.0;
+    if (i < B) {
+        unsigned blk = warp;
+        for (; blk + 7 * NT_WARPS < nblk; blk += 8 * NT_WARPS) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldcg(partials + (int64_t)(blk + u * NT_WARPS) * B + i);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) t += (double)v[u];
+        }
+        for (; blk < nblk; blk += NT_WARPS) t += (double)__ldcg(partials + (int64_t)blk * B + i);
+    }
+    comb[warp][lane] = t;
+    __syncthreads();
+    double r = 0.0;
+    if (warp == 0) {
+#pragma unroll
+        for (int w = 0; w < NT_WARPS; ++w) r += comb[w][lane];
+    }
+    __syncthreads();
+    return r;
+}
+
 // ---------------------------------------------------------------------------------
 // one-pass norm test
 // ---------------------------------------------------------------------------------
@@ -357,12 +387,15 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
     __threadfence();
 
     // last block: combine all partials in a fixed order, in fp64
+    __shared__ double smem_comb[NT_WARPS][32];
     double q_local = 0.0;
-    for (int64_t i = tid; i < B; i += NT_THREADS) {
-        double t = 0.0;
-        for (unsigned blk = 0; blk < gridDim.x; ++blk) t += (double)__ldcg(a.n_partials + (int64_t)blk * B + i);
-        if (a.n_out != nullptr) a.n_out[i] = a.n_accum ? a.n_out[i] + (float)t : (float)t;
-        q_local += t;
+    for (int64_t i0 = 0; i0 < B; i0 += 32) {
+        const double t = combine_rows32(a.n_partials, B, gridDim.x, i0, smem_comb);
+        const int64_t i = i0 + lane;
+        if (warp == 0 && i < B) {
+            if (a.n_out != nullptr) a.n_out[i] = a.n_accum ? a.n_out[i] + (float)t : (float)t;
+            q_local += t;
+        }
     }
     double p0 = 0.0, p1 = 0.0, p2 = 0.0;
     for (unsigned blk = tid; blk < gridDim.x; blk += NT_THREADS) {
@@ -632,14 +665,17 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) centred_dot_kerne
     const adloco_test_sums s = *a.sums;
     const double bd = (double)B;
     const double N = s.sum_sq_gsum / (bd * bd);
+    __shared__ double smem_comb[NT_WARPS][32];
     double l_d2 = 0.0, l_d = 0.0;
-    for (int64_t i = tid; i < B; i += NT_THREADS) {
-        double t = 0.0;
-        for (unsigned blk = 0; blk < gridDim.x; ++blk) t += (double)__ldcg(a.n_partials + (int64_t)blk * B + i);
-        const double d = t / bd;
-        if (a.dots_out != nullptr) a.dots_out[i] = (float)(N + d);
-        l_d2 += d * d;
-        l_d += d;
+    for (int64_t i0 = 0; i0 < B; i0 += 32) {
+        const double t = combine_rows32(a.n_partials, B, gridDim.x, i0, smem_comb);
+        const int64_t i = i0 + (tid & 31);
+        if ((tid >> 5) == 0 && i < B) {
+            const double d = t / bd;
+            if (a.dots_out != nullptr) a.dots_out[i] = (float)(N + d);
+            l_d2 += d * d;
+            l_d += d;
+        }
     }
     const double sum_d2 = block_sum(l_d2, smem_red);
     const double sum_d = block_sum(l_d, smem_red);
