@@ -975,14 +975,26 @@ __device__ __forceinline__ void outer_update(float th, float v, double acc, cons
 // Every thread owns four consecutive elements per iteration: theta and v arrive as
 // one 128-bit load each, an instance as 128 bits (fp32) or 64 bits (bf16), so all
 // accesses of a warp are contiguous and every fetched sector is used in full.
+// four consecutive elements of an instance as they sit in memory (64 bits of bf16 or 128
+// bits of fp32): kept packed in registers until used, so that KB loads in flight cost
+// 2 KB registers for bf16 instances instead of 4 KB
 template <bool BF16>
-__device__ __forceinline__ void load_inst4(const void* base, int64_t i, float (&x)[4]) {
+struct InstRaw {
+    typename std::conditional<BF16, uint2, float4>::type w;
+};
+template <bool BF16>
+__device__ __forceinline__ InstRaw<BF16> load_inst4(const void* base, int64_t i) {
+    InstRaw<BF16> r;
+    if constexpr (BF16) r.w = __ldcs(reinterpret_cast<const uint2*>(base) + i);
+    else r.w = __ldcs(reinterpret_cast<const float4*>(base) + i);
+    return r;
+}
+template <bool BF16>
+__device__ __forceinline__ void unpack_inst4(const InstRaw<BF16>& r, float (&x)[4]) {
     if constexpr (BF16) {
-        const uint2 w = __ldcs(reinterpret_cast<const uint2*>(base) + i);
-        x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
+        x[0] = bf16_lo(r.w.x); x[1] = bf16_hi(r.w.x); x[2] = bf16_lo(r.w.y); x[3] = bf16_hi(r.w.y);
     } else {
-        const float4 w = __ldcs(reinterpret_cast<const float4*>(base) + i);
-        x[0] = w.x; x[1] = w.y; x[2] = w.z; x[3] = w.w;
+        x[0] = r.w.x; x[1] = r.w.y; x[2] = r.w.z; x[3] = r.w.w;
     }
 }
 
@@ -990,11 +1002,17 @@ __device__ __forceinline__ void load_inst4(const void* base, int64_t i, float (&
 // when there are at least 8 instances, else 4 (6 blocks per SM) -- measured: K=8 runs 3 %
 // faster with the former, K=4 5 % faster with the latter.
 template <bool BF16, bool WB, int KB>
-__global__ void __launch_bounds__(256, KB == 8 ? 4 : 6) outer_step_kernel(const __grid_constant__ OuterArgs a) {
+__global__ void __launch_bounds__(256, (KB == 8 && !BF16) ? 3 : 4) outer_step_kernel(const __grid_constant__ OuterArgs a) {
     constexpr int VEC = 4;
     const int64_t nvec = a.P / VEC;
     const int64_t step = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
+        // all loads of the element group are issued before anything is used: the first KB instances,
+        // then theta and v (a use of theta ahead of the instance loads costs a second memory round trip)
+        InstRaw<BF16> x[KB];
+#pragma unroll
+        for (int u = 0; u < KB; ++u)
+            if (u < a.K) x[u] = load_inst4<BF16>(a.inst[u], i);
         const float4 t4 = __ldcs(reinterpret_cast<const float4*>(a.th_in) + i);
         const float4 v4 = __ldcs(reinterpret_cast<const float4*>(a.v_in) + i);
         const float th[VEC] = {t4.x, t4.y, t4.z, t4.w};
@@ -1002,21 +1020,26 @@ __global__ void __launch_bounds__(256, KB == 8 ? 4 : 6) outer_step_kernel(const 
         double acc[VEC], thd[VEC];
 #pragma unroll
         for (int e = 0; e < VEC; ++e) { acc[e] = 0.0; thd[e] = (double)th[e]; }
-        int k = 0;
-        for (; k + KB <= a.K; k += KB) {
-            float x[KB][VEC];
 #pragma unroll
-            for (int u = 0; u < KB; ++u) load_inst4<BF16>(a.inst[k + u], i, x[u]);
+        for (int u = 0; u < KB; ++u)
+            if (u < a.K) {
+                float xe[VEC];
+                unpack_inst4<BF16>(x[u], xe);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[e] += thd[e] - (double)xe[e];
+            }
+        for (int k = KB; k < a.K; k += KB) {
 #pragma unroll
             for (int u = 0; u < KB; ++u)
+                if (k + u < a.K) x[u] = load_inst4<BF16>(a.inst[k + u], i);
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) acc[e] += thd[e] - (double)x[u][e];
-        }
-        for (; k < a.K; ++k) {
-            float x[VEC];
-            load_inst4<BF16>(a.inst[k], i, x);
+            for (int u = 0; u < KB; ++u)
+                if (k + u < a.K) {
+                    float xe[VEC];
+                    unpack_inst4<BF16>(x[u], xe);
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) acc[e] += thd[e] - (double)x[e];
+                    for (int e = 0; e < VEC; ++e) acc[e] += thd[e] - (double)xe[e];
+                }
         }
         float tn[VEC], vn[VEC];
 #pragma unroll
@@ -1122,9 +1145,10 @@ __global__ void __launch_bounds__(256) pseudo_grad_kernel(const float* __restric
     const int64_t nvec = P / 4;
     const int64_t step = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
+        const InstRaw<BF16> raw = load_inst4<BF16>(inst, i);
         const float4 t = __ldcs(reinterpret_cast<const float4*>(theta) + i);
         float x[4];
-        load_inst4<BF16>(inst, i, x);
+        unpack_inst4<BF16>(raw, x);
         __stcs(reinterpret_cast<float4*>(g) + i, make_float4(t.x - x[0], t.y - x[1], t.z - x[2], t.w - x[3]));
     }
     if (blockIdx.x == 0) {
