@@ -101,9 +101,9 @@ def aggregate_throughput(units_per_rank: float, world: int, max_seconds: float) 
 
 
 # DRAM traffic of norm_test_kernel per gradient element, from the ncu capture of the
-# profiling case (B=64, P=2^21: 537.0 MB read + 1.63 MB written for 2^27 elements);
+# profiling case (B=64, P=2^21: 537.0 MB read + 7.0 MB written for 2^27 elements);
 # traffic grows in proportion to B*P, so a full launch is this times its element count.
-NT_TRAFFIC_BYTES_PER_ELEMENT = (537.0e6 + 1.63e6) / float(64 * (1 << 21))
+NT_TRAFFIC_BYTES_PER_ELEMENT = (537.0e6 + 7.0e6) / float(64 * (1 << 21))
 # DRAM traffic of the grouped direct kernel (CTA-pair form) per transformer block of four
 # layers at B=32, T=1024, from the ncu capture of the profiling case (one block: 902.3 MB
 # read + 24.0 MB written for 805.3 MB of operands); every block's operands are read once,
@@ -607,6 +607,21 @@ def run_table(args):
         ts.sort()
         return ts[len(ts) // 2]
 
+    def gpu_ms_rotating(fns, rounds=10):
+        """Throughput of a small kernel: the calls in `fns` (the same kernel on different buffers, together
+        larger than L2) run back to back for `rounds` rounds with no synchronisation in between."""
+        for fn in fns:
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(rounds):
+            for fn in fns:
+                fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (rounds * len(fns))
+
     def cpu_s(fn):
         t0 = time.perf_counter()
         fn()
@@ -648,7 +663,17 @@ def run_table(args):
     emit(1, "norm_test (B=16, P=2^20)", ms, nbytes=4 * 16 * (1 << 20), oracle_s=cpu_s(lambda: O.norm_test(Gn, eta=0.5)),
          oracle_note="whole", note="L2 flushed between repetitions; launch-latency bound")
     outer_case(1, 4, 1 << 20, torch.float32)
-    del G
+    # the same two kernels back to back over four rotating input sets (256 MB / 134 MB in all, more than L2):
+    # throughput without the launch latency a lone call pays
+    Gs = [W.per_sample_grads(16, 1 << 20, seed=100 + r, device=dev) for r in range(4)]
+    ms = gpu_ms_rotating([(lambda g=g: ctx.norm_test(g, p, sync=False)) for g in Gs])
+    emit(1, "norm_test (B=16, P=2^20), back to back over 4 rotating inputs", ms, nbytes=4 * 16 * (1 << 20),
+         note="throughput; the row above is the latency of one call")
+    states = [W.outer_state(4, 1 << 20, inst_dtype=torch.float32, seed=200 + r, device=dev) for r in range(4)]
+    ms = gpu_ms_rotating([(lambda st=st: ctx.outer_step(st[1], st[0], st[2], lr=LR, momentum=MU)) for st in states])
+    emit(1, "outer_step (K=4 fp32, P=1048576), back to back over 4 rotating states", ms, nbytes=(4 * 4 + 16) * (1 << 20),
+         note="throughput; the row above is the latency of one call")
+    del G, Gs, states
     # config 2
     G = W.per_sample_grads(NT_B, 1 << 24, seed=2, device=dev)
     p = A.make_params(0.1, b_cur=64, b_max=32)
@@ -687,11 +712,21 @@ def run_table(args):
     emit(3, "linear_sqnorm direct (norms + gradient sum)", ms_d, flops=mg, oracle_s=o_s, oracle_note="whole",
          note="same outputs as the row above from one GEMM")
     emit(3, "linear_sqnorm pair (CTA-pair direct kernel)", ms_p, flops=mg, oracle_s=o_s, oracle_note="whole")
+    ms_gp = gpu_ms(lambda: ctx.linear_sqnorm(X, D, n, method="gram_pair"))
+    emit(3, "gram_pair (Gram identity over CTA pairs, norms only)", ms_gp, flops=sym,
+         note="40 of 128x128 sub-blocks computed per sample for 36 needed")
     Sb = torch.zeros(GR_DOUT, device=dev)
     ms_b = gpu_ms(lambda: ctx.vector_param_sqnorm(D, n, grad_sum=Sb), flush=True)
     Dn8 = Dn[:8]
     emit(3, "vector_param_sqnorm (bias of the layer, Delta [32,1024,3072])", ms_b, nbytes=2 * GR_B * GR_T * GR_DOUT,
          oracle_s=cpu_s(lambda: O.vector_param_terms(Dn8)) * 4, oracle_note="8 samples timed, x4", note="L2 flushed")
+    # throughput of the same kernel back to back (no L2 flush needed: the 201 MB operand exceeds L2, and
+    # two operands alternate)
+    D2 = D.clone()
+    ms_b2 = gpu_ms_rotating([lambda: ctx.vector_param_sqnorm(D, n, grad_sum=Sb), lambda: ctx.vector_param_sqnorm(D2, n, grad_sum=Sb)])
+    emit(3, "vector_param_sqnorm, back to back over 2 alternating operands", ms_b2, nbytes=2 * GR_B * GR_T * GR_DOUT,
+         note="throughput; the row above is the latency of one call after an L2 flush")
+    del D2
     gen = torch.Generator(device=dev)
     gen.manual_seed(4)
     ids = torch.randint(0, 50257, (GR_B, GR_T), generator=gen, device=dev, dtype=torch.int32)
