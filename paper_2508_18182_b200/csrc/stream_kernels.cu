@@ -282,7 +282,10 @@ __device__ __forceinline__ void nt_row_tile(const elem_t* rowp, int64_t stride, 
 // squares of (G_ij - G_0j) -- shifting by the first row removes the mean before
 // squaring, so the centred sum of squares comes out without cancellation -- and
 // per row the running sum of squares (RB registers, rows tiled by RB).
-template <int RB, bool VEC, bool BF16 = false>
+// MICRO = switch-mode accumulation (a.mode == NT_MICRO), an instantiation of its own: the running sums it
+// fetches and the term of the pairwise update cost registers that the one-shot form, at 64 rows per thread,
+// does not have (with them in, the row loop spilled and ran 9 % slower, 14 % under the power cap).
+template <int RB, bool VEC, bool BF16 = false, bool MICRO = false>
 __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(const __grid_constant__ NtArgs a) {
     using elem_t = typename std::conditional<BF16, __nv_bfloat16, float>::type;
     constexpr int CH = RB < NT_CHUNK ? RB : NT_CHUNK;   // rows loaded back to back
@@ -302,14 +305,17 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
     const float Bf = (float)B;
     const float invB = 1.0f / Bf;
     // switch-mode accumulation: samples already accumulated before this micro-batch
-    const double c_prev_d = (a.mode == NT_MICRO) ? (double)a.sums->batch_count : 0.0;
+    const double c_prev_d = MICRO ? (double)a.sums->batch_count : 0.0;
     const float inv_cprev = c_prev_d > 0.0 ? (float)(1.0 / c_prev_d) : 0.f;
 
     float acc[RB];
 #pragma unroll
     for (int r = 0; r < RB; ++r) acc[r] = 0.f;
 
-    double t_sumsq = 0.0, t_css = 0.0, t_chan = 0.0;
+    // per-thread fp64 running sums live in shared memory (touched once per 16 column groups): as registers
+    // they pushed the 64-row instantiation into spilling inside the row loop
+    __shared__ double smem_run[3][NT_THREADS];
+    smem_run[0][tid] = 0.0; smem_run[1][tid] = 0.0; smem_run[2][tid] = 0.0;
     float f_sumsq = 0.f, f_css = 0.f, f_chan = 0.f;
 
     for (int it = 0; it < a.iters; ++it) {
@@ -323,7 +329,7 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
         float4 sd = c, sdd = c;
         // switch mode: the sums so far are fetched now, so that their latency hides behind the rows
         float4 so = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (a.mode == NT_MICRO && nvalid > 0) so = load4<VEC>(a.S + col, nvalid);
+        if (MICRO && nvalid > 0) so = load4<VEC>(a.S + col, nvalid);
         for (int64_t i0 = 0; i0 < B; i0 += RB) {
             if (nvalid == 4 && i0 + RB <= B)
                 nt_row_tile<RB, CH, VEC, false>(rowp, a.stride, RB, 4, i0 == 0, c, sd, sdd, acc);
@@ -342,7 +348,7 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
         s.x = fmaf(Bf, c.x, sd.x); s.y = fmaf(Bf, c.y, sd.y); s.z = fmaf(Bf, c.z, sd.z); s.w = fmaf(Bf, c.w, sd.w);
         f_css += (sdd.x - sd.x * sd.x * invB) + (sdd.y - sd.y * sd.y * invB) +
                  (sdd.z - sd.z * sd.z * invB) + (sdd.w - sd.w * sd.w * invB);
-        if (a.mode == NT_MICRO) {
+        if (MICRO) {
             // pairwise (Chan) update of the centred sum of squares needs ||mean_mb - mean_prev||^2
             const float ex = s.x * invB - so.x * inv_cprev, ey = s.y * invB - so.y * inv_cprev;
             const float ez = s.z * invB - so.z * inv_cprev, ew = s.w * invB - so.w * inv_cprev;
@@ -354,11 +360,13 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
         }
         f_sumsq += s.x * s.x + s.y * s.y + s.z * s.z + s.w * s.w;
         if ((it & 15) == 15) {  // bound the length of the fp32 running sums
-            t_sumsq += (double)f_sumsq; t_css += (double)f_css; t_chan += (double)f_chan;
+            smem_run[0][tid] += (double)f_sumsq; smem_run[1][tid] += (double)f_css;
+            if (MICRO) smem_run[2][tid] += (double)f_chan;
             f_sumsq = f_css = f_chan = 0.f;
         }
     }
-    t_sumsq += (double)f_sumsq; t_css += (double)f_css; t_chan += (double)f_chan;
+    const double t_sumsq = smem_run[0][tid] + (double)f_sumsq, t_css = smem_run[1][tid] + (double)f_css;
+    const double t_chan = smem_run[2][tid] + (double)f_chan;
     if (single_tile) warp_rows_flush<RB>(acc, my_rows, lane);
 
     // block partials
@@ -444,13 +452,13 @@ static int grow_workspace(adloco_ctx* ctx, size_t need_elems) {
     return ADLOCO_OK;
 }
 
-template <int RB, bool VEC, bool BF16>
+template <int RB, bool VEC, bool BF16, bool MICRO>
 static int launch_nt(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
     const int64_t ngroups = (l.P + 3) / 4;
     const int64_t tiles = (ngroups + NT_THREADS - 1) / NT_THREADS;
     const int Bpad = (int)(((l.B + RB - 1) / RB) * RB);
     const size_t smem = (size_t)NT_WARPS * Bpad * sizeof(float);
-    auto kern = norm_test_kernel<RB, VEC, BF16>;
+    auto kern = norm_test_kernel<RB, VEC, BF16, MICRO>;
     if (smem > 48 * 1024) ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // resident blocks per SM for this instantiation and shared-memory size (asked once)
     static std::mutex cache_mutex;            // contexts on different host threads share these statics
@@ -492,16 +500,20 @@ int launch_norm_test(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
     const uintptr_t row_align = l.bf16 ? 7u : 15u;
     const bool vec = (reinterpret_cast<uintptr_t>(l.G) & row_align) == 0 && (l.B == 1 || (l.stride % 4) == 0) &&
                      (l.S == nullptr || aligned16(l.S));
-#define ADLOCO_NT_DISPATCH(V, H)                                         \
+#define ADLOCO_NT_DISPATCH(V, H, M)                                      \
     do {                                                                 \
-        if (l.B <= 4) return launch_nt<4, V, H>(ctx, l, st);             \
-        if (l.B <= 8) return launch_nt<8, V, H>(ctx, l, st);             \
-        if (l.B <= 16) return launch_nt<16, V, H>(ctx, l, st);           \
-        if (l.B <= 32) return launch_nt<32, V, H>(ctx, l, st);           \
-        return launch_nt<64, V, H>(ctx, l, st);                          \
+        if (l.B <= 4) return launch_nt<4, V, H, M>(ctx, l, st);          \
+        if (l.B <= 8) return launch_nt<8, V, H, M>(ctx, l, st);          \
+        if (l.B <= 16) return launch_nt<16, V, H, M>(ctx, l, st);        \
+        if (l.B <= 32) return launch_nt<32, V, H, M>(ctx, l, st);        \
+        return launch_nt<64, V, H, M>(ctx, l, st);                       \
     } while (0)
-    if (l.bf16) { if (vec) ADLOCO_NT_DISPATCH(true, true); else ADLOCO_NT_DISPATCH(false, true); }
-    if (vec) ADLOCO_NT_DISPATCH(true, false); else ADLOCO_NT_DISPATCH(false, false);
+    if (l.mode == NT_MICRO) {
+        if (l.bf16) { if (vec) ADLOCO_NT_DISPATCH(true, true, true); else ADLOCO_NT_DISPATCH(false, true, true); }
+        if (vec) ADLOCO_NT_DISPATCH(true, false, true); else ADLOCO_NT_DISPATCH(false, false, true);
+    }
+    if (l.bf16) { if (vec) ADLOCO_NT_DISPATCH(true, true, false); else ADLOCO_NT_DISPATCH(false, true, false); }
+    if (vec) ADLOCO_NT_DISPATCH(true, false, false); else ADLOCO_NT_DISPATCH(false, false, false);
 #undef ADLOCO_NT_DISPATCH
 }
 
