@@ -599,6 +599,37 @@ __device__ void ip_decide_device(double sum_d2, double sum_d, const adloco_test_
 // their entries of S once and walks down the rows accumulating, per row,
 // sum_j (G_ij - S_j / b) S_j = b (<g_i, gbar> - ||gbar||^2): centring before the
 // product keeps the small deviation d_i free of cancellation.
+// One tile of RB rows for the inner-product pass, as nt_row_tile does for the norm test: CHECKED = false
+// (a full tile of a full column group) has no guards, so a chunk's loads stay in flight together.
+template <int RB, int CH, bool VEC, bool CHECKED, typename elem_t>
+__device__ __forceinline__ void ip_row_tile(const elem_t* rowp, int64_t stride, int64_t rows_left, int nvalid,
+                                            float invB, const float4& s4, float (&acc)[RB]) {
+    float4 m4;
+#pragma unroll
+    for (int r0 = 0; r0 < RB; r0 += CH) {
+        float4 x[CH];
+#pragma unroll
+        for (int u = 0; u < CH; ++u) {
+            if (CHECKED) x[u] = load4<VEC>(rowp + (int64_t)(r0 + u) * stride, (r0 + u) < rows_left ? nvalid : 0);
+            else x[u] = load4<VEC>(rowp + (int64_t)(r0 + u) * stride, 4);
+        }
+        // the column means are formed from the sums only now: a use of s4 ahead of the first chunk's loads
+        // would hold those loads back by one memory round trip
+        if (r0 == 0) m4 = make_float4(s4.x * invB, s4.y * invB, s4.z * invB, s4.w * invB);
+#pragma unroll
+        for (int u = 0; u < CH; ++u) {
+            if (!CHECKED || (r0 + u) < rows_left) {
+                // columns beyond P carry s4 = 0 and add nothing
+                float q = (x[u].x - m4.x) * s4.x;
+                q = fmaf(x[u].y - m4.y, s4.y, q);
+                q = fmaf(x[u].z - m4.z, s4.z, q);
+                q = fmaf(x[u].w - m4.w, s4.w, q);
+                acc[r0 + u] += q;
+            }
+        }
+    }
+}
+
 template <int RB, bool VEC, bool BF16 = false>
 __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) centred_dot_kernel(const __grid_constant__ IpArgs a) {
     using elem_t = typename std::conditional<BF16, __nv_bfloat16, float>::type;
@@ -628,28 +659,11 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) centred_dot_kerne
         if (g < ngroups) nvalid = (a.P - col) >= 4 ? 4 : (int)(a.P - col);
         const elem_t* rowp = reinterpret_cast<const elem_t*>(a.G) + (nvalid > 0 ? col : 0);
         const float4 s4 = load4<VEC>(a.S + (nvalid > 0 ? col : 0), nvalid);
-        const float4 m4 = make_float4(s4.x * invB, s4.y * invB, s4.z * invB, s4.w * invB);
         for (int64_t i0 = 0; i0 < B; i0 += RB) {
-#pragma unroll
-            for (int r0 = 0; r0 < RB; r0 += CH) {
-                float4 x[CH];
-#pragma unroll
-                for (int u = 0; u < CH; ++u) {
-                    const bool ok = (i0 + r0 + u) < B;
-                    x[u] = load4<VEC>(rowp + (int64_t)(r0 + u) * a.stride, ok ? nvalid : 0);
-                }
-#pragma unroll
-                for (int u = 0; u < CH; ++u) {
-                    if ((i0 + r0 + u) < B) {
-                        // columns beyond P carry s4 = 0 and add nothing
-                        float q = (x[u].x - m4.x) * s4.x;
-                        q = fmaf(x[u].y - m4.y, s4.y, q);
-                        q = fmaf(x[u].z - m4.z, s4.z, q);
-                        q = fmaf(x[u].w - m4.w, s4.w, q);
-                        acc[r0 + u] += q;
-                    }
-                }
-            }
+            if (nvalid == 4 && i0 + RB <= B)
+                ip_row_tile<RB, CH, VEC, false>(rowp, a.stride, RB, 4, invB, s4, acc);
+            else
+                ip_row_tile<RB, CH, VEC, true>(rowp, a.stride, B - i0, nvalid, invB, s4, acc);
             rowp += (int64_t)RB * a.stride;
             if (!single_tile) {
                 warp_rows_flush<RB>(acc, my_rows + i0, lane);
