@@ -830,6 +830,19 @@ def run_table(args):
     out = torch.empty_like(inst[0])
     ms = gpu_ms(lambda: ctx.merge(inst, [3, 17, 5, 8], out))
     emit("merge", "adloco_merge (K=4 bf16, P=124,439,808)", ms, nbytes=(2 * 4 + 2) * W.GPT2_SMALL_P)
+    # the three kernels of the outer step with one instance per GPU (the exchange between them needs several GPUs
+    # and is not timed here): one rank's share at the GPT-2-small size, its slice of a world of 8 for the update
+    P = W.GPT2_SMALL_P
+    theta, inst, mom = W.outer_state(1, P, inst_dtype=torch.bfloat16, seed=11, device=dev)
+    g = torch.empty(P, device=dev)
+    ms = gpu_ms(lambda: ctx.pseudo_gradient(theta, inst[0], g))
+    emit("exchange form", "adloco_pseudo_gradient (bf16 instance, P=124,439,808)", ms, nbytes=(4 + 2 + 4) * P)
+    L = P // 8
+    ms = gpu_ms(lambda: ctx.outer_apply(g[:L], 8, theta[:L], mom[:L], lr=LR, momentum=MU), flush=True)
+    emit("exchange form", "adloco_outer_apply (one rank's slice of 8, P/8 elements)", ms, nbytes=(4 + 8 + 8) * L,
+         note="L2 flushed; 311 MB per call")
+    ms = gpu_ms(lambda: ctx.refresh_instance(theta, inst[0]))
+    emit("exchange form", "adloco_refresh_instance (bf16 instance, P=124,439,808)", ms, nbytes=(4 + 2) * P)
     ctx.close()
 
 
