@@ -263,6 +263,12 @@ int adloco_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
  *   ADLOCO_LINEAR_DIRECT_PAIR  the direct route with 256 x 256 tiles, each shared by the two
  *                         SMs of a thread-block cluster (each loads half of the operands);
  *                         ADLOCO_ERR_UNSUPPORTED where cluster launches are not available.
+ *   ADLOCO_LINEAR_GRAM_ONE_CTA / ADLOCO_LINEAR_GRAM_PAIR  the Gram identity by a named kernel: one CTA
+ *                         per 128 x 256-token tile (what ADLOCO_LINEAR_GRAM and adloco_gram_sqnorm run), or
+ *                         256 x 256-token tiles shared by the two SMs of a cluster (same result; a third less
+ *                         traffic into shared memory and one read of the operands from HBM, for one unused
+ *                         128 x 128 sub-block per diagonal tile; measured as fast as the one-CTA kernel at
+ *                         T = 1024; ADLOCO_ERR_UNSUPPORTED where cluster launches are not available).
  *   ADLOCO_LINEAR_AUTO    whichever executes fewer tensor-core flops for the shape
  *                         (direct wins when T exceeds about d_in d_out / (d_in + d_out));
  *                         the direct route then runs in its pair form where available. */

@@ -296,7 +296,7 @@ static int gram_route(adloco_ctx* ctx, const void* X, const void* D, int64_t B, 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (variant == 1 && !pair_launch_ok(ctx)) return ADLOCO_ERR_UNSUPPORTED;
     if (variant < 0) variant = 0;
-    int rc = variant == 1 ? launch_gram_pair(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, 1, st)
+    int rc = variant == 1 ? launch_gram_pair(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, st)
                           : launch_gram_sqnorm(ctx, X, D, B, T, d_in, d_out, per_sample_sqnorm, accumulate_norms, st);
     if (rc != ADLOCO_OK) return rc;
     if (grad_sum) rc = launch_mean_grad(ctx, X, D, B, T, d_in, d_out, grad_sum, accumulate_sum, st);

@@ -166,7 +166,7 @@ int launch_accum_sqnorm(adloco_ctx* ctx, adloco_accum* acc, cudaStream_t st);
 int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                        int64_t d_out, float* n, int accumulate_norms, cudaStream_t st);
 int launch_gram_pair(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
-                     int64_t d_out, float* n, int accumulate_norms, int with_diag, cudaStream_t st);
+                     int64_t d_out, float* n, int accumulate_norms, cudaStream_t st);
 int launch_mean_grad(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
                      int64_t d_out, float* S, int accumulate_sum, cudaStream_t st);
 int launch_embedding(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, int64_t T, int64_t d, int64_t V,

@@ -287,8 +287,7 @@ struct GramPairArgs {
     int B, T, d_in, d_out;
     int nt;               // 128-token blocks per side
     int m;                // 256-token blocks per side
-    int rects;            // items per sample: m (m + 1) / 2, or m (m - 1) / 2 when the diagonal is left out
-    int with_diag;        // 0: only items with q > p
+    int rects;            // items per sample: m (m + 1) / 2
     int total_items;
     int* counter;         // zero at launch
     float* n;             // [B], +=
@@ -299,13 +298,12 @@ struct GramPairArgs {
 __device__ __forceinline__ void gram_pair_decode(int item, const GramPairArgs& a, int& i, int& p, int& q) {
     i = item / a.rects;
     int r = item - i * a.rects;
-    const int first = a.with_diag ? 0 : 1;        // offset of the first block column of a row from its diagonal
-    for (p = 0; p < a.m - 1; ++p) {
-        const int cnt = a.m - p - first;
+    for (p = 0; p < a.m - 1; ++p) {         // block row p has the m - p block columns p .. m - 1
+        const int cnt = a.m - p;
         if (r < cnt) break;
         r -= cnt;
     }
-    q = p + first + r;
+    q = p + r;
 }
 
 __global__ void __launch_bounds__(GP_THREADS, 1)
@@ -1502,9 +1500,9 @@ int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B,
     return ADLOCO_OK;
 }
 
-// The CTA-pair form of the Gram kernel; with_diag = 0 leaves the 256-token blocks on the diagonal out
+// The CTA-pair form of the Gram kernel
 int launch_gram_pair(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,
-                     int64_t d_out, float* n, int accumulate_norms, int with_diag, cudaStream_t st) {
+                     int64_t d_out, float* n, int accumulate_norms, cudaStream_t st) {
     CUtensorMap tmX, tmD;
     int rc = cached_map(ctx, &tmX, X, B, T, d_in, GR_TILE);
     if (rc != ADLOCO_OK) return rc;
@@ -1514,14 +1512,12 @@ int launch_gram_pair(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
     a.B = (int)B; a.T = (int)T; a.d_in = (int)d_in; a.d_out = (int)d_out;
     a.nt = (int)((T + GR_TILE - 1) / GR_TILE);
     a.m = (a.nt + 1) / 2;
-    const int64_t rects = with_diag ? (int64_t)a.m * (a.m + 1) / 2 : (int64_t)a.m * (a.m - 1) / 2;
+    const int64_t rects = (int64_t)a.m * (a.m + 1) / 2;
     if (rects * B > 0x3fffffff) return ADLOCO_ERR_UNSUPPORTED;
     a.rects = (int)rects;
-    a.with_diag = with_diag;
     a.total_items = (int)(rects * B);
     a.n = n; a.status = ctx->gemm_status; a.wait_ns = ctx->wait_limit_ns;
     if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
-    if (a.total_items == 0) return ADLOCO_OK;
     a.counter = ctx->sched_counters + (ctx->sched_next.fetch_add(1) % kSchedCounters);
     ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(a.counter, 0, sizeof(int), st));
     static std::atomic<bool> attr_set[64];   // the attribute is per device
