@@ -317,8 +317,12 @@ int adloco_vector_param_sqnorm(adloco_ctx* ctx, const void* D, const void* X, in
 
 /* Per-sample gradient norms of an embedding table E [V, d] looked up at every token
  * (Eq. 1 applied to E): row v of sample i's gradient is the sum of delta_{i,t} over the
- * tokens with token_ids[i, t] = v, so n_i = sum_{t,s} [id_t == id_s] (delta_t . delta_s)
- * -- the Gram identity with a token-equality mask in place of X X^T, on the tensor cores.
+ * tokens with token_ids[i, t] = v, and n_i = sum_v || sum_{t: id_t = v} delta_t ||^2.
+ * Up to T = 4096 the tokens of a sample are grouped by id on chip and every delta row is
+ * read once (a streaming pass; ids that occur once contribute their row's squared norm,
+ * repeated ids the squared norm of their rows' sum); longer sequences take the equivalent
+ * n_i = sum_{t,s} [id_t == id_s] (delta_t . delta_s) -- the Gram identity with a
+ * token-equality mask in place of X X^T -- on the tensor cores.
  * With position indices as ids it covers a learned positional embedding.
  *   token_ids          dev int32 [B, T], values in [0, V) (others match nothing and are skipped)
  *   D                  dev bf16 [B, T, d]: gradient of the loss w.r.t. the looked-up rows; d % 8 == 0

@@ -5,10 +5,17 @@
 //                       for every tile on or above the diagonal of the token-by-token
 //                       Gram matrices both products are accumulated in TMEM and the
 //                       epilogue reduces their elementwise product.
+//   gram_pair_kernel    the same over pairs of CTAs (cta_group::2, 256-token tiles).
 //   mean_grad_kernel    S (+)= sum_i D_i^T X_i, the batch gradient sum, a GEMM whose
 //                       contraction runs over all tokens of all samples.
+//   direct_group_kernel every sample's weight-gradient tile formed in TMEM (norms and the
+//                       gradient sum from one GEMM), over groups of layers, one CTA or a
+//                       pair of CTAs per tile.
+//   embed_gram_kernel / embed_segment_kernel / embed_scatter_kernel: embedding tables
+//                       (the segment and scatter kernels are plain streaming kernels; they
+//                       sit here beside the masked Gram form of the same norms).
 //
-// Both are persistent, warp-specialised kernels: warp 0 issues TMA tile loads
+// The tensor-core kernels are persistent and warp-specialised: warp 0 issues TMA tile loads
 // into a ring of shared-memory stages, warp 1 issues tcgen05.mma from shared
 // memory into TMEM accumulators, the remaining warps drain the accumulators.
 // Every wait is bounded; a wait that runs out raises a status word and all
@@ -692,6 +699,252 @@ embed_gram_kernel(const __grid_constant__ CUtensorMap tmD, const EmbedArgs ea) {
         tmem_dealloc(tmem_base, 512);
     }
     if (threadIdx.x == 0 && abort_flag) atomicExch(a.status, (int)ADLOCO_ERR_TIMEOUT);
+}
+
+// =====================================================================================
+// embedding norms by grouping: the streaming form
+// =====================================================================================
+// ||G_i||^2 = sum over the table rows v of || sum_{t: id_t = v} delta_t ||^2 needs every delta row once:
+// B T d reads against the B T^2 d flops of the masked Gram sum above, which stays as the route for
+// sequences longer than ES_MAX_T.  Written as  sum_t ||delta_t||^2  +  sum over the ids that occur more
+// than once of ( ||sum of their rows||^2 - sum of their ||.||^2 ):  the first term is a plain stream over
+// all rows, the second touches only the rows of repeated ids (again; they are in L2).  Each block of
+// sample i groups the sample's T tokens by id in shared memory -- an open-addressing table of H >= 2T
+// slots, a count per slot, a prefix sum, a scatter: the tokens of one id end up next to each other in
+// `order` -- streams its share of the rows, and sums the groups that start at its share of the
+// positions: a warp per group, lane = 8 features per 256; groups of more than ES_BIG rows are summed by
+// all warps of the block together.  All blocks of a sample build the same table (T atomics in shared
+// memory: cheap next to the rows), so nothing passes through global memory between them.
+constexpr int ES_WARPS = 16;
+constexpr int ES_THREADS = 32 * ES_WARPS;
+constexpr int ES_MAX_T = 4096;          // (3 H + 4 T) ints of shared memory: 160 KB at T = 4096
+constexpr int ES_BIG = 64;              // rows from which a group is summed by the whole block
+constexpr int ES_NF = 2;                // feature chunks of 256 a warp carries per pass over a small group
+constexpr int ES_MAX_BIG = ES_MAX_T / ES_BIG;
+
+struct EmbedSegArgs {
+    const int* ids;                 // [B, T]
+    const __nv_bfloat16* D;         // [B, T, d]
+    int T, d, V, H, chunks;         // H: power of two >= 2 T; chunks: blocks per sample
+    float* n;                       // [B], +=
+};
+
+__device__ __forceinline__ void es_add_row(float (&acc)[8], const uint4& w) {
+    acc[0] += __uint_as_float(w.x << 16); acc[1] += __uint_as_float(w.x & 0xffff0000u);
+    acc[2] += __uint_as_float(w.y << 16); acc[3] += __uint_as_float(w.y & 0xffff0000u);
+    acc[4] += __uint_as_float(w.z << 16); acc[5] += __uint_as_float(w.z & 0xffff0000u);
+    acc[6] += __uint_as_float(w.w << 16); acc[7] += __uint_as_float(w.w & 0xffff0000u);
+}
+
+__global__ void __launch_bounds__(ES_THREADS, 2) embed_segment_kernel(const EmbedSegArgs a) {
+    extern __shared__ int es_smem[];
+    int* keys = es_smem;             // [H] id held by the slot, -1 = free
+    int* cnt = keys + a.H;           // [H] tokens of that id
+    int* start = cnt + a.H;          // [H] first position of the id's group in `order`
+    int* slot_of = start + a.H;      // [T] slot of token t, -1 = id outside the table
+    int* rank = slot_of + a.T;       // [T] arrival number of token t within its group
+    int* order = rank + a.T;         // [T] token indices, grouped by id
+    int* glen = order + a.T;         // [T] length of the group that starts at this position, else 0
+    __shared__ float part[ES_WARPS][256];
+    __shared__ int big_list[ES_MAX_BIG];
+    __shared__ int n_big;
+    __shared__ int scan_warp[ES_WARPS];
+    __shared__ double red[ES_WARPS];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int i = blockIdx.y, c = blockIdx.x;
+    const int T = a.T, H = a.H, d = a.d;
+    const int* ids_i = a.ids + (int64_t)i * T;
+    const __nv_bfloat16* D_i = a.D + (int64_t)i * T * d;
+
+    for (int s = tid; s < H; s += ES_THREADS) { keys[s] = -1; cnt[s] = 0; }
+    for (int t = tid; t < T; t += ES_THREADS) glen[t] = 0;
+    if (tid == 0) n_big = 0;
+    __syncthreads();
+    // every token finds the slot of its id (the first to arrive claims it) and takes a number
+    for (int t = tid; t < T; t += ES_THREADS) {
+        const int id = __ldg(ids_i + t);
+        int slot = -1;
+        if (id >= 0 && id < a.V) {
+            slot = (int)(((uint32_t)id * 2654435761u) & (uint32_t)(H - 1));
+            for (;;) {
+                const int prev = atomicCAS(&keys[slot], -1, id);
+                if (prev == -1 || prev == id) break;
+                slot = (slot + 1) & (H - 1);       // H >= 2 T slots: a free one always turns up
+            }
+            rank[t] = atomicAdd(&cnt[slot], 1);
+        }
+        slot_of[t] = slot;
+    }
+    __syncthreads();
+    // exclusive prefix sum of the counts: each thread owns H / ES_THREADS consecutive slots (H is a power of two)
+    {
+        const int per = H >= ES_THREADS ? H / ES_THREADS : 1;
+        const int s0 = tid * per;
+        int local = 0;
+        if (s0 < H)
+            for (int k = 0; k < per; ++k) local += cnt[s0 + k];
+        int incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) scan_warp[warp] = incl;
+        __syncthreads();
+        int base = 0;
+        for (int w = 0; w < warp; ++w) base += scan_warp[w];
+        int run = base + incl - local;
+        if (s0 < H)
+            for (int k = 0; k < per; ++k) { start[s0 + k] = run; run += cnt[s0 + k]; }
+    }
+    __syncthreads();
+    for (int t = tid; t < T; t += ES_THREADS) {
+        const int slot = slot_of[t];
+        if (slot >= 0) {
+            const int p0 = start[slot];
+            order[p0 + rank[t]] = t;
+            if (rank[t] == 0) glen[p0] = cnt[slot];
+        }
+    }
+    __syncthreads();
+
+    // (A) every token inside the table adds ||delta_t||^2: the block streams its share of the rows, eight
+    // rows in flight per warp.  For an id that occurs once this is the whole contribution.
+    float sa = 0.f;
+    {
+        const int rows_per = (T + a.chunks - 1) / a.chunks;
+        const int t_lo = c * rows_per;
+        const int t_hi = t_lo + rows_per < T ? t_lo + rows_per : T;
+        for (int fc = 0; fc < d; fc += 256) {
+            const int f = fc + lane * 8;
+            if (f >= d) break;                                   // the same for every later fc too
+            for (int t = t_lo + warp; t < t_hi; t += 8 * ES_WARPS) {
+                uint4 w[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int tt = t + u * ES_WARPS;
+                    w[u] = make_uint4(0, 0, 0, 0);
+                    if (tt < t_hi && slot_of[tt] >= 0) w[u] = __ldcs(reinterpret_cast<const uint4*>(D_i + (int64_t)tt * d + f));
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float r[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    es_add_row(r, w[u]);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) sa = fmaf(r[e], r[e], sa);
+                }
+            }
+        }
+    }
+    // (B) an id that occurs L >= 2 times adds ||sum of its rows||^2 - sum of their ||.||^2 on top (twice the
+    // inner products between its rows).  Groups of up to ES_BIG rows: one warp each; the group that starts
+    // at position p belongs to warp p % ES_WARPS of block (p / ES_WARPS) % chunks.
+    double sq = 0.0;
+    for (int p = c * ES_WARPS + warp; p < T; p += a.chunks * ES_WARPS) {
+        const int L = glen[p];
+        if (L < 2) continue;
+        if (L > ES_BIG) {
+            if (lane == 0) big_list[atomicAdd(&n_big, 1)] = p;     // at most T / ES_BIG of them
+            continue;
+        }
+        for (int fc = 0; fc < d; fc += 256 * ES_NF) {
+            float acc[ES_NF][8];
+#pragma unroll
+            for (int j = 0; j < ES_NF; ++j)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
+            float own = 0.f;                                     // sum of the rows' own squared norms
+            for (int r = 0; r < L; r += 2) {
+                const int t0 = order[p + r];
+                const int t1 = (r + 1 < L) ? order[p + r + 1] : -1;
+                uint4 w0[ES_NF], w1[ES_NF];
+#pragma unroll
+                for (int j = 0; j < ES_NF; ++j) {
+                    const int f = fc + j * 256 + lane * 8;
+                    w0[j] = make_uint4(0, 0, 0, 0);
+                    w1[j] = make_uint4(0, 0, 0, 0);
+                    if (f < d) {
+                        w0[j] = __ldg(reinterpret_cast<const uint4*>(D_i + (int64_t)t0 * d + f));
+                        if (t1 >= 0) w1[j] = __ldg(reinterpret_cast<const uint4*>(D_i + (int64_t)t1 * d + f));
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < ES_NF; ++j) {
+                    float r0[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, r1[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    es_add_row(r0, w0[j]);
+                    es_add_row(r1, w1[j]);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        own = fmaf(r0[e], r0[e], own);
+                        own = fmaf(r1[e], r1[e], own);
+                        acc[j][e] += r0[e] + r1[e];
+                    }
+                }
+            }
+            float s2 = 0.f;
+#pragma unroll
+            for (int j = 0; j < ES_NF; ++j)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) s2 = fmaf(acc[j][e], acc[j][e], s2);
+            sq += (double)s2 - (double)own;
+        }
+    }
+    __syncthreads();
+    // long groups (a frequent token, padding that maps inside the table): all warps of the block share
+    // the rows of one group; their partial sums meet in shared memory before they are squared
+    const int nb = n_big;
+    for (int k = 0; k < nb; ++k) {
+        const int p = big_list[k];
+        const int L = glen[p];
+        for (int fc = 0; fc < d; fc += 256) {
+            const int f = fc + lane * 8;
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+            float own = 0.f;
+            if (f < d) {
+                for (int r = warp; r < L; r += 4 * ES_WARPS) {
+                    uint4 w[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int rr = r + u * ES_WARPS;
+                        w[u] = make_uint4(0, 0, 0, 0);
+                        if (rr < L) w[u] = __ldg(reinterpret_cast<const uint4*>(D_i + (int64_t)order[p + rr] * d + f));
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        float r8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                        es_add_row(r8, w[u]);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) { own = fmaf(r8[e], r8[e], own); acc[e] += r8[e]; }
+                    }
+                }
+            }
+            sq -= (double)own;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) part[warp][lane * 8 + e] = acc[e];
+            __syncthreads();
+            if (tid < 256) {
+                float g = 0.f;
+#pragma unroll
+                for (int w = 0; w < ES_WARPS; ++w) g += part[w][tid];
+                sq += (double)g * (double)g;
+            }
+            __syncthreads();
+        }
+    }
+    sq += (double)sa;
+    // block total -> n_i
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if (lane == 0) red[warp] = sq;
+    __syncthreads();
+    if (tid == 0) {
+        double tot = 0.0;
+        for (int w = 0; w < ES_WARPS; ++w) tot += red[w];
+        if (tot != 0.0) atomicAdd(a.n + i, (float)tot);
+    }
 }
 
 // S[id_t, :] += delta_t for every token: one warp per token row, 128-bit loads, vector reductions
@@ -1542,8 +1795,50 @@ int launch_gram_pair(adloco_ctx* ctx, const void* X, const void* D, int64_t B, i
     return ADLOCO_OK;
 }
 
+// the scatter-add of the gradient sum, shared by both routes of the norms
+static int launch_embed_scatter(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, int64_t T, int64_t d, int64_t V,
+                                float* S, int accumulate_sum, cudaStream_t st) {
+    if (!accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)V * (size_t)d * sizeof(float), st));
+    const int64_t tokens = B * T;
+    int64_t blocks = (tokens + 7) / 8;
+    const int64_t cap = (int64_t)ctx->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    embed_scatter_kernel<<<(unsigned)blocks, 256, 0, st>>>(ids, static_cast<const __nv_bfloat16*>(D), tokens, (int)d, (int)V, S);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
 int launch_embedding(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, int64_t T, int64_t d, int64_t V,
                      float* n, int accumulate_norms, float* S, int accumulate_sum, cudaStream_t st) {
+    if (T <= ES_MAX_T && B <= 65535) {
+        // the streaming form: every delta row read once
+        EmbedSegArgs ea;
+        ea.ids = ids; ea.D = static_cast<const __nv_bfloat16*>(D);
+        ea.T = (int)T; ea.d = (int)d; ea.V = (int)V; ea.n = n;
+        int H = 64;
+        while (H < 2 * T) H <<= 1;
+        ea.H = H;
+        int64_t chunks = (2 * (int64_t)ctx->sm_count) / B;             // all blocks resident at once, two per SM
+        const int64_t most = (T + ES_WARPS - 1) / ES_WARPS;
+        if (chunks > most) chunks = most;
+        if (chunks > 32) chunks = 32;
+        if (chunks < 1) chunks = 1;
+        ea.chunks = (int)chunks;
+        const size_t smem = ((size_t)3 * H + (size_t)4 * T) * sizeof(int);
+        if (!accumulate_norms) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(n, 0, (size_t)B * sizeof(float), st));
+        static std::atomic<bool> attr_set[64];   // the attribute is per device
+        if (!attr_set[ctx->device & 63].load()) {
+            ADLOCO_CUDA_TRY(ctx, cudaFuncSetAttribute(embed_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                      (int)(((size_t)3 * 2 * ES_MAX_T + (size_t)4 * ES_MAX_T) * sizeof(int))));
+            attr_set[ctx->device & 63].store(true);
+        }
+        embed_segment_kernel<<<dim3((unsigned)chunks, (unsigned)B), ES_THREADS, smem, st>>>(ea);
+        ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+        ctx->launches++;
+        if (S) return launch_embed_scatter(ctx, ids, D, B, T, d, V, S, accumulate_sum, st);
+        return ADLOCO_OK;
+    }
     CUtensorMap tmD;
     int rc = cached_map(ctx, &tmD, D, B, T, d, GR_TILE);
     if (rc != ADLOCO_OK) return rc;
@@ -1572,17 +1867,7 @@ int launch_embedding(adloco_ctx* ctx, const int* ids, const void* D, int64_t B, 
     embed_gram_kernel<<<grid, GR_THREADS, GR_SMEM, st>>>(tmD, ea);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
-    if (S) {
-        if (!accumulate_sum) ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(S, 0, (size_t)V * (size_t)d * sizeof(float), st));
-        const int64_t tokens = B * T;
-        int64_t blocks = (tokens + 7) / 8;
-        const int64_t cap = (int64_t)ctx->sm_count * 8;
-        if (blocks > cap) blocks = cap;
-        embed_scatter_kernel<<<(unsigned)blocks, 256, 0, st>>>(ids, static_cast<const __nv_bfloat16*>(D), tokens, (int)d,
-                                                               (int)V, S);
-        ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
-        ctx->launches++;
-    }
+    if (S) return launch_embed_scatter(ctx, ids, D, B, T, d, V, S, accumulate_sum, st);
     return ADLOCO_OK;
 }
 

@@ -1,6 +1,8 @@
 """GPU parity: adloco_embedding_sqnorm (per-sample gradient norms of an embedding
-table through the Gram identity with a token-equality mask; scatter-added gradient
-sum) against the oracle, which scatters every sample's gradient explicitly."""
+table -- by grouping a sample's tokens by id and summing each group's rows, or, for
+sequences beyond 4096 tokens, through the Gram identity with a token-equality mask;
+scatter-added gradient sum) against the oracle, which scatters every sample's gradient
+explicitly."""
 import numpy as np
 import pytest
 import torch
@@ -28,7 +30,11 @@ def _ids(B, T, V, seed):
 
 
 @pytest.mark.parametrize("B,T,d,V", [(3, 7, 8, 5), (4, 128, 64, 20), (2, 300, 72, 40), (5, 1024, 768, 1000),
-                                     (3, 257, 136, 3), (1, 1, 8, 1), (6, 513, 256, 50257)])
+                                     (3, 257, 136, 3), (1, 1, 8, 1), (6, 513, 256, 50257),
+                                     (2, 4096, 72, 300),     # the longest sequence the grouping kernel takes (160 KB of shared memory)
+                                     (1, 4100, 64, 50),      # beyond it: the masked Gram kernel
+                                     (40, 96, 1048, 7),      # d > 1024: several feature passes; groups of ~14 rows
+                                     (2, 900, 264, 4)])      # groups of > 64 rows: summed by the whole block
 def test_matches_oracle(ctx, B, T, d, V):
     _, D = W.linear_layer(B, T, 8, d, seed=B + T, delta_std=1.0, device=DEV)
     ids = _ids(B, T, V, seed=d)

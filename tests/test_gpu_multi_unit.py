@@ -85,9 +85,9 @@ def test_config3_layer_direct_route_full_size(ctx):
     _check_layer(ctx, X, D, "gram_pair", "config 3 Gram over CTA pairs")
 
 
-def test_embedding_with_several_items_per_cta(ctx):
-    """B=32, T=1024, d=768: 640 work items on 148 CTAs, so each CTA alternates between its two
-    accumulator buffers four or five times."""
+def test_embedding_at_full_size(ctx):
+    """B=32, T=1024, d=768 with a 2000-row table (about 230 ids per sample occur more than once),
+    then with three ids only (groups of ~340 rows, summed block-wide)."""
     B, T, d, V = 32, 1024, 768, 2000
     _, D = W.linear_layer(B, T, 8, d, seed=17, delta_std=1.0, device=DEV)
     g = torch.Generator(device=DEV)
@@ -101,12 +101,29 @@ def test_embedding_with_several_items_per_cta(ctx):
     n_ref, S_ref = O.embedding_terms(ids.cpu().numpy(), W.to_numpy(D), V)
     assert np.allclose(n.cpu().numpy(), n_ref, rtol=TOL_BF16), (n.cpu().numpy() / n_ref)
     assert np.allclose(S.cpu().numpy(), S_ref, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(S_ref).max() * 0.05)
-    # few distinct ids: most token pairs match, the masked sum is dense
+    # few distinct ids: three long groups per sample
     ids2 = torch.randint(0, 3, (B, T), generator=g, device=DEV, dtype=torch.int32)
     ctx.embedding_sqnorm(ids2, D, V, n)
     torch.cuda.synchronize()
     n_ref2, _ = O.embedding_terms(ids2.cpu().numpy(), W.to_numpy(D), V)
     assert np.allclose(n.cpu().numpy(), n_ref2, rtol=TOL_BF16)
+
+
+def test_embedding_gram_kernel_with_several_items_per_cta(ctx):
+    """Sequences beyond 4096 tokens go through the masked Gram kernel: B=2, T=4352 gives 34 blocks
+    per side, 306 + 17 work items per sample on 148 CTAs, so each CTA alternates between its two
+    accumulator buffers four or five times."""
+    B, T, d, V = 2, 4352, 128, 900
+    _, D = W.linear_layer(B, T, 8, d, seed=19, delta_std=1.0, device=DEV)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(20)
+    ids = torch.randint(0, V, (B, T), generator=g, device=DEV, dtype=torch.int32)
+    n = torch.full((B,), -1.0, device=DEV)
+    ctx.embedding_sqnorm(ids, D, V, n)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    n_ref, _ = O.embedding_terms(ids.cpu().numpy(), W.to_numpy(D), V)
+    assert np.allclose(n.cpu().numpy(), n_ref, rtol=TOL_BF16), (n.cpu().numpy() / n_ref)
 
 
 # ---------------------------------------------------------------- groups of layers in one launch
