@@ -21,9 +21,9 @@
  *     legacy default stream) and is asynchronous unless stated.  The streaming
  *     entry points (norm test, accumulate, finalize, inner-product test, host
  *     variants) share the ctx workspace: do not run two of them at the same
- *     time on one ctx.  The tensor-core entry points (adloco_gram_sqnorm,
- *     adloco_linear_sqnorm, adloco_embedding_sqnorm), adloco_vector_param_sqnorm,
- *     adloco_outer_step and adloco_merge use none of it and may be issued on
+ *     time on one ctx.  The per-layer entry points (adloco_gram_sqnorm,
+ *     adloco_linear_sqnorm, adloco_linear_sqnorm_group, adloco_embedding_sqnorm,
+ *     adloco_vector_param_sqnorm), adloco_outer_step and adloco_merge use none of it and may be issued on
  *     several streams at once -- the layers of one micro-batch only add into
  *     n and into their own S, and alternating them on two streams overlaps
  *     one kernel's tail with the next one's start.
