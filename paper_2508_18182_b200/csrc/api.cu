@@ -44,6 +44,19 @@ int ensure_staging(adloco_ctx* ctx, size_t bytes_each) {
 
 constexpr size_t kPanelBytes = 64u << 20;  // staging panel of the host-memory entry points
 
+// The device-side address of a caller's host buffer when the GPU can store to it directly (page-locked
+// memory under unified addressing), else null: a result struct then goes there from the deciding thread
+// itself and the stream is spared a device-to-host copy between two kernels.  Pageable memory gets the copy.
+static void* device_address_of_pinned(void* host) {
+    if (!host) return nullptr;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 // thread-block clusters of two CTAs need compute capability 9.0 or later and the launch attribute
 bool pair_launch_ok(adloco_ctx* ctx) {
     if (ctx->pair_ok < 0) {
@@ -176,9 +189,10 @@ int adloco_norm_test(adloco_ctx* ctx, const void* grads, adloco_dtype dtype, int
     l.n_out = per_sample_sqnorm; l.S = grad_sum;
     l.sums = sums_dev ? sums_dev : ctx->scratch_sums;
     l.result = result_dev; l.params = *params; l.mode = NT_ONESHOT;
+    l.result_mirror = static_cast<adloco_test_result*>(device_address_of_pinned(result_host));
     rc = launch_norm_test(ctx, l, st);
     if (rc != ADLOCO_OK) return rc;
-    if (result_host)
+    if (result_host && !l.result_mirror)
         ADLOCO_CUDA_TRY(ctx, cudaMemcpyAsync(result_host, result_dev, sizeof(adloco_test_result), cudaMemcpyDeviceToHost, st));
     return ADLOCO_OK;
 }
@@ -190,9 +204,10 @@ int adloco_test_decide(adloco_ctx* ctx, const adloco_test_sums* sums_dev, const 
     if (rc != ADLOCO_OK) return rc;
     DeviceGuard g(ctx->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = launch_decide(ctx, sums_dev, *params, result_dev, st);
+    adloco_test_result* mirror = static_cast<adloco_test_result*>(device_address_of_pinned(result_host));
+    rc = launch_decide(ctx, sums_dev, *params, result_dev, mirror, st);
     if (rc != ADLOCO_OK) return rc;
-    if (result_host)
+    if (result_host && !mirror)
         ADLOCO_CUDA_TRY(ctx, cudaMemcpyAsync(result_host, result_dev, sizeof(adloco_test_result), cudaMemcpyDeviceToHost, st));
     return ADLOCO_OK;
 }
@@ -272,9 +287,10 @@ int adloco_inner_product_test(adloco_ctx* ctx, const void* grads, adloco_dtype d
     l.bf16 = (dtype == ADLOCO_BF16);
     l.S = grad_sum; l.B = B; l.P = P; l.stride = row_stride; l.sums = sums_dev; l.params = *params;
     l.dots_out = inner_products; l.result = result_dev;
+    l.result_mirror = static_cast<adloco_ip_result*>(device_address_of_pinned(result_host));
     rc = launch_inner_product(ctx, l, st);
     if (rc != ADLOCO_OK) return rc;
-    if (result_host)
+    if (result_host && !l.result_mirror)
         ADLOCO_CUDA_TRY(ctx, cudaMemcpyAsync(result_host, result_dev, sizeof(adloco_ip_result), cudaMemcpyDeviceToHost, st));
     return ADLOCO_OK;
 }
@@ -506,11 +522,12 @@ int adloco_accum_finalize(adloco_ctx* ctx, adloco_accum* a, const adloco_test_pa
         if (rc != ADLOCO_OK) return rc;
         a->sqnorm_current = true;
     }
-    rc = launch_decide(ctx, a->state, *params, result_dev, st);
+    adloco_test_result* mirror = static_cast<adloco_test_result*>(device_address_of_pinned(result_host));
+    rc = launch_decide(ctx, a->state, *params, result_dev, mirror, st);
     if (rc != ADLOCO_OK) return rc;
     if (sums_dev)
         ADLOCO_CUDA_TRY(ctx, cudaMemcpyAsync(sums_dev, a->state, sizeof(adloco_test_sums), cudaMemcpyDeviceToDevice, st));
-    if (result_host)
+    if (result_host && !mirror)
         ADLOCO_CUDA_TRY(ctx, cudaMemcpyAsync(result_host, result_dev, sizeof(adloco_test_result), cudaMemcpyDeviceToHost, st));
     return ADLOCO_OK;
 }

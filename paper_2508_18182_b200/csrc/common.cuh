@@ -103,13 +103,14 @@ struct NtLaunch {
     float* S = nullptr;           // [P]: written (ONESHOT/PANEL) or read-modify-written (MICRO); may be null unless MICRO
     adloco_test_sums* sums = nullptr;    // required (ctx scratch if the caller has none)
     adloco_test_result* result = nullptr;  // decision written by the last block when non-null
+    adloco_test_result* result_mirror = nullptr;  // device-side address of a page-locked host copy of it, or null
     adloco_test_params params{};
     int mode = NT_ONESHOT;
     int first_panel = 1;          // PANEL: overwrite the sums on the first panel, add afterwards
 };
 int launch_norm_test(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st);
 int launch_decide(adloco_ctx* ctx, const adloco_test_sums* sums, const adloco_test_params& p,
-                  adloco_test_result* result, cudaStream_t st);
+                  adloco_test_result* result, adloco_test_result* mirror, cudaStream_t st);
 
 struct IpLaunch {
     const float* G = nullptr;
@@ -120,6 +121,7 @@ struct IpLaunch {
     adloco_ip_params params{};
     float* dots_out = nullptr;
     adloco_ip_result* result = nullptr;
+    adloco_ip_result* result_mirror = nullptr;
 };
 int launch_inner_product(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st);
 

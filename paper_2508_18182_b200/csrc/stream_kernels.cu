@@ -135,7 +135,10 @@ __device__ __forceinline__ void warp_rows_flush(float (&v)[RB], float* dst, int 
 // ---------------------------------------------------------------------------------
 // batch rule + switch plan (Section "Norm test", Section "Mode switching")
 // ---------------------------------------------------------------------------------
-__device__ void decide_device(const adloco_test_sums& s, const adloco_test_params& p, adloco_test_result* out) {
+// `mirror`, when given, is the caller's page-locked host copy of the result: the deciding thread stores
+// there too, which spares the stream a device-to-host copy between two kernels (about 11 us per call).
+__device__ void decide_device(const adloco_test_sums& s, const adloco_test_params& p, adloco_test_result* out,
+                              adloco_test_result* mirror = nullptr) {
     adloco_test_result r;
     const int64_t b = s.batch_count;
     const double bd = (double)b;
@@ -186,10 +189,15 @@ __device__ void decide_device(const adloco_test_sums& s, const adloco_test_param
         r.b_micro = r.b_req < p.b_max ? r.b_req : p.b_max;
     }
     *out = r;
+    if (mirror != nullptr) {
+        *mirror = r;
+        __threadfence_system();
+    }
 }
 
-__global__ void decide_kernel(const adloco_test_sums* sums, adloco_test_params p, adloco_test_result* out) {
-    if (threadIdx.x == 0 && blockIdx.x == 0) decide_device(*sums, p, out);
+__global__ void decide_kernel(const adloco_test_sums* sums, adloco_test_params p, adloco_test_result* out,
+                              adloco_test_result* mirror) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) decide_device(*sums, p, out, mirror);
 }
 
 // Last block of a reduction: the total over all blocks of the per-block partial sums of 32
@@ -235,6 +243,7 @@ struct NtArgs {
     float* S;
     adloco_test_sums* sums;
     adloco_test_result* result;
+    adloco_test_result* result_mirror;   // page-locked host copy the last block also writes, or null
     adloco_test_params params;
     float* n_partials;
     double* blk_scalars;
@@ -432,7 +441,7 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) norm_test_kernel(
             s.batch_count += B;
         }
         *a.sums = s;
-        if (a.result != nullptr) decide_device(s, a.params, a.result);
+        if (a.result != nullptr) decide_device(s, a.params, a.result, a.result_mirror);
         *a.ticket = 0u;
     }
 }
@@ -486,7 +495,7 @@ static int launch_nt(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
 
     NtArgs a;
     a.G = l.G; a.B = l.B; a.P = l.P; a.stride = l.stride;
-    a.n_out = l.n_out; a.S = l.S; a.sums = l.sums; a.result = l.result; a.params = l.params;
+    a.n_out = l.n_out; a.S = l.S; a.sums = l.sums; a.result = l.result; a.result_mirror = l.result_mirror; a.params = l.params;
     a.n_partials = ctx->n_partials; a.blk_scalars = ctx->blk_scalars; a.ticket = ctx->ticket;
     a.mode = l.mode; a.n_accum = l.n_accum; a.first_panel = l.first_panel; a.iters = (int)iters;
     kern<<<(unsigned)grid, NT_THREADS, smem, st>>>(a);
@@ -518,8 +527,8 @@ int launch_norm_test(adloco_ctx* ctx, const NtLaunch& l, cudaStream_t st) {
 }
 
 int launch_decide(adloco_ctx* ctx, const adloco_test_sums* sums, const adloco_test_params& p,
-                  adloco_test_result* result, cudaStream_t st) {
-    decide_kernel<<<1, 32, 0, st>>>(sums, p, result);
+                  adloco_test_result* result, adloco_test_result* mirror, cudaStream_t st) {
+    decide_kernel<<<1, 32, 0, st>>>(sums, p, result, mirror);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     return ADLOCO_OK;
@@ -536,6 +545,7 @@ struct IpArgs {
     adloco_ip_params params;
     float* dots_out;           // [B] <g_i, gbar>, may be null
     adloco_ip_result* result;
+    adloco_ip_result* result_mirror;   // page-locked host copy, or null
     float* n_partials;
     unsigned* ticket;
     int iters;
@@ -707,6 +717,10 @@ __global__ void __launch_bounds__(NT_THREADS, RB <= 8 ? 4 : 2) centred_dot_kerne
     const double sum_d = block_sum(l_d, smem_red);
     if (tid == 0) {
         ip_decide_device(sum_d2, sum_d, s, a.params, a.result);
+        if (a.result_mirror != nullptr) {
+            *a.result_mirror = *a.result;
+            __threadfence_system();
+        }
         *a.ticket = 0u;
     }
 }
@@ -743,7 +757,7 @@ static int launch_ip_t(adloco_ctx* ctx, const IpLaunch& l, cudaStream_t st) {
     if (rc != ADLOCO_OK) return rc;
     IpArgs a;
     a.G = l.G; a.S = l.S; a.B = l.B; a.P = l.P; a.stride = l.stride; a.sums = l.sums; a.params = l.params;
-    a.dots_out = l.dots_out; a.result = l.result;
+    a.dots_out = l.dots_out; a.result = l.result; a.result_mirror = l.result_mirror;
     a.n_partials = ctx->n_partials; a.ticket = ctx->ticket; a.iters = (int)iters;
     kern<<<(unsigned)grid, NT_THREADS, smem, st>>>(a);
     ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
@@ -954,7 +968,7 @@ int adloco_norm_test_noalloc(const float* grads, int64_t B, int64_t P, int64_t r
     a.blk_scalars = reinterpret_cast<double*>(base + NA_PARTIALS_BYTES);
     a.ticket = reinterpret_cast<unsigned*>(base + NA_PARTIALS_BYTES + NA_SCALARS_BYTES);
     a.sums = reinterpret_cast<adloco_test_sums*>(base + NA_PARTIALS_BYTES + NA_SCALARS_BYTES + 256);
-    a.result = result_dev; a.params = *params;
+    a.result = result_dev; a.result_mirror = nullptr; a.params = *params;
     a.mode = NT_ONESHOT; a.n_accum = 0; a.first_panel = 1; a.iters = 0;
     // the array keeps whatever the last call left: the ticket must start at zero
     if (cudaMemsetAsync(a.ticket, 0, NA_TAIL_BYTES, st) != cudaSuccess) return ADLOCO_ERR_CUDA;

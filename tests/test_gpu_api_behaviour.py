@@ -73,3 +73,35 @@ def test_empty_inputs_are_argument_errors_and_launch_nothing():
     assert lib.adloco_merge(h, arr, w, A.F32, 1, 16, d, None, None) == A.ERR_INVALID_ARG      # weight 0
     assert c.launch_count == before
     c.close()
+
+
+def test_host_copy_of_the_result_in_page_locked_and_in_pageable_memory():
+    """result_host in page-locked memory is written by the kernel itself; in pageable memory it is
+    filled by a copy on the stream.  Both hold the decision once the stream is synchronised, for
+    the norm test, the re-decision from stored sums and the accumulator's final test."""
+    import ctypes as C
+    import oracle.adloco_oracle as O
+    from parity import TOL_F32, assert_test_result
+    c = A.Context(0)
+    G = W.per_sample_grads(16, (1 << 16) + 4, sigma=0.5, seed=1, device=DEV)
+    p = A.make_params(0.5, b_cur=16, b_max=32)
+    ora = O.norm_test(W.to_numpy(G), eta=0.5, b_cur=16, b_max=32)
+    pinned = c.norm_test(G, p)                                       # the binding's page-locked buffer
+    pageable = A.TestResult()
+    vp = C.c_void_p
+    rc = c.lib.adloco_norm_test(c.h, vp(G.data_ptr()), A.F32, 16, G.shape[1], G.stride(0), C.byref(p), None, None,
+                                vp(c._sums_dev.data_ptr()), vp(c._res_dev.data_ptr()), C.cast(C.byref(pageable), vp), None)
+    assert rc == 0
+    torch.cuda.synchronize()
+    assert_test_result(pinned, ora, p, TOL_F32, what="page-locked result")
+    assert (pageable.stat, pageable.b_req, pageable.flags, pageable.sum_sqnorm) == (pinned.stat, pinned.b_req, pinned.flags, pinned.sum_sqnorm)
+    p2 = A.make_params(1.0, b_cur=16, b_max=32)
+    again = c.test_decide(p2)
+    pageable2 = A.TestResult()
+    rc = c.lib.adloco_test_decide(c.h, vp(c._sums_dev.data_ptr()), C.byref(p2), vp(c._res_dev.data_ptr()), C.cast(C.byref(pageable2), vp), None)
+    assert rc == 0
+    torch.cuda.synchronize()
+    o2 = O.decide(ora.sum_sqnorm, ora.mean_sqnorm, ora.variance, 16, eta=1.0, b_cur=16, b_max=32)
+    assert_test_result(again, o2, p2, TOL_F32, what="re-decision")
+    assert (pageable2.stat, pageable2.b_req) == (again.stat, again.b_req)
+    c.close()
