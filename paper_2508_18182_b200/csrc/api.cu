@@ -477,9 +477,8 @@ int adloco_accum_reset(adloco_ctx* ctx, adloco_accum* a, void* stream) {
     if (!ctx || !a || a->ctx != ctx) return ADLOCO_ERR_INVALID_ARG;
     DeviceGuard g(ctx->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    for (int i = 0; i < a->n_bufs; ++i)
-        ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(a->bufs_host[i], 0, (size_t)a->sizes_host[i] * sizeof(float), st));
-    ADLOCO_CUDA_TRY(ctx, cudaMemsetAsync(a->state, 0, sizeof(adloco_test_sums), st));
+    const int rc = launch_accum_zero(ctx, a, st);     // every S buffer and the state, one launch
+    if (rc != ADLOCO_OK) return rc;
     a->sqnorm_current = true;
     return ADLOCO_OK;
 }

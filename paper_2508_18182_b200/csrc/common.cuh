@@ -163,6 +163,7 @@ int launch_merge(adloco_ctx* ctx, const MergeLaunch& l, cudaStream_t st);
 // state->sum_sqnorm += sum(n[0..b)) and the count (form (b) of adloco_accumulate)
 int launch_accum_add_norms(adloco_ctx* ctx, adloco_accum* acc, const float* n, int64_t b, cudaStream_t st);
 int launch_accum_sqnorm(adloco_ctx* ctx, adloco_accum* acc, cudaStream_t st);
+int launch_accum_zero(adloco_ctx* ctx, adloco_accum* acc, cudaStream_t st);
 
 // ---- tensor-core path, implemented in gram_kernels.cu ---------------------------
 int launch_gram_sqnorm(adloco_ctx* ctx, const void* X, const void* D, int64_t B, int64_t T, int64_t d_in,

@@ -1441,6 +1441,45 @@ __global__ void __launch_bounds__(256) accum_sqnorm_kernel(float* const* bufs, c
     }
 }
 
+// All gradient-sum buffers of the accumulator and its state set to zero in one launch (a model's
+// accumulator has one buffer per parameter: a memset each would put dozens of tiny operations on the stream).
+__global__ void __launch_bounds__(256) accum_zero_kernel(float* const* bufs, const int64_t* sizes, const int64_t* chunk_prefix,
+                                                         int n_bufs, int64_t total_chunks, adloco_test_sums* state) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        adloco_test_sums z;
+        memset(&z, 0, sizeof(z));
+        *state = z;
+    }
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t ch = blockIdx.x; ch < total_chunks; ch += gridDim.x) {
+        int lo = 0, hi = n_bufs - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (chunk_prefix[mid] <= ch) lo = mid; else hi = mid - 1;
+        }
+        float* base = bufs[lo];
+        const int64_t size = sizes[lo];
+        const int64_t off = (ch - chunk_prefix[lo]) * SQ_CHUNK;
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const int64_t j = off + ((int64_t)h * 256 + threadIdx.x) * 4;
+            if (j < size) store4(base + j, zero, (size - j) >= 4 ? 4 : (int)(size - j));
+        }
+    }
+}
+
+int launch_accum_zero(adloco_ctx* ctx, adloco_accum* acc, cudaStream_t st) {
+    int64_t grid = acc->total_chunks;
+    const int64_t cap = (int64_t)ctx->sm_count * 8;
+    if (grid > cap) grid = cap;
+    if (grid < 1) grid = 1;
+    accum_zero_kernel<<<(unsigned)grid, 256, 0, st>>>(acc->bufs_dev, acc->sizes_dev, acc->chunk_prefix_dev, acc->n_bufs,
+                                                     acc->total_chunks, acc->state);
+    ADLOCO_CUDA_TRY(ctx, cudaGetLastError());
+    ctx->launches++;
+    return ADLOCO_OK;
+}
+
 int launch_accum_sqnorm(adloco_ctx* ctx, adloco_accum* acc, cudaStream_t st) {
     int64_t grid = acc->total_chunks;
     const int64_t cap = (int64_t)ctx->sm_count * 8;
