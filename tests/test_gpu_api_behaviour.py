@@ -39,6 +39,45 @@ def test_non_default_stream_and_two_contexts():
     c2.close()
 
 
+def test_layers_of_one_micro_batch_on_two_streams_add_into_the_same_norms():
+    """The per-layer entry points use no context workspace: layers issued alternately on two streams
+    (every route, an embedding and a bias among them) add into one n vector atomically and each into
+    its own sum buffer; every launch that draws work from a counter gets a counter of its own."""
+    c = A.Context(0)
+    s = [torch.cuda.Stream(), torch.cuda.Stream()]
+    B, T = 6, 384
+    shapes = [(128, 256), (256, 128), (64, 512), (512, 64), (128, 128), (256, 256), (72, 264), (264, 72)]
+    methods = ["pair", "gram_pair", "direct", "gram", "auto", "pair", "gram_pair", "direct"]
+    data = [W.linear_layer(B, T, di, do, seed=40 + l, device=DEV) for l, (di, do) in enumerate(shapes)]
+    sums = [torch.full((do, di), 9.0, device=DEV) for di, do in shapes]
+    g = torch.Generator(device=DEV)
+    g.manual_seed(7)
+    ids = torch.randint(0, 50, (B, T), generator=g, device=DEV, dtype=torch.int32)
+    n = torch.zeros(B, device=DEV)
+    Sb = torch.full((256,), 9.0, device=DEV)
+    torch.cuda.synchronize()
+    for l, ((X, D), S, m) in enumerate(zip(data, sums, methods)):
+        with torch.cuda.stream(s[l & 1]):
+            c.linear_sqnorm(X, D, n, accumulate_norms=True, grad_sum=S, method=m, stream=s[l & 1])
+    with torch.cuda.stream(s[0]):
+        c.embedding_sqnorm(ids, data[0][1], 50, n, accumulate_norms=True, stream=s[0])
+    with torch.cuda.stream(s[1]):
+        c.vector_param_sqnorm(data[0][1], n, accumulate_norms=True, grad_sum=Sb, stream=s[1])
+    torch.cuda.synchronize()
+    assert c.device_status() == 0
+    n_ref = np.zeros(B)
+    for (X, D), S in zip(data, sums):
+        n_l, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
+        n_ref += n_l
+        assert np.allclose(S.cpu().numpy(), S_ref, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(S_ref).max() * 0.05)
+    n_ref += O.embedding_terms(ids.cpu().numpy(), W.to_numpy(data[0][1]), 50)[0]
+    nb, Sb_ref = O.vector_param_terms(W.to_numpy(data[0][1]))
+    n_ref += nb
+    assert np.allclose(n.cpu().numpy(), n_ref, rtol=TOL_BF16), n.cpu().numpy() / n_ref
+    assert np.allclose(Sb.cpu().numpy(), Sb_ref, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(Sb_ref).max() * 0.05)
+    c.close()
+
+
 def test_bad_device_index_is_an_error_not_a_crash():
     with pytest.raises(A.AdlocoError) as e:
         A.Context(4096)
