@@ -79,12 +79,12 @@ def test_linear_layer_random_shapes(ctx):
     rng = np.random.default_rng(99)
     for case in range(24):
         B = int(rng.integers(1, 9))
-        T = int(rng.integers(1, 400))
+        T = int(rng.integers(1, 400)) if case % 4 else int(rng.integers(400, 1300))
         d_in = 8 * int(rng.integers(1, 50))
         d_out = 8 * int(rng.integers(1, 70))
         X, D = W.linear_layer(B, T, d_in, d_out, seed=case, delta_std=0.1, device=DEV)
         n_ref, S_ref = O.linear_layer_terms(W.to_numpy(X), W.to_numpy(D))
-        for method in ("gram", "direct"):
+        for method in ("gram", "gram_pair", "direct", "pair"):
             n = torch.zeros(B, device=DEV)
             S = torch.zeros(d_out, d_in, device=DEV)
             ctx.linear_sqnorm(X, D, n, grad_sum=S, method=method)
@@ -100,4 +100,12 @@ def test_linear_layer_random_shapes(ctx):
         torch.cuda.synchronize()
         nb_ref, Sb_ref = O.vector_param_terms(W.to_numpy(Dg), W.to_numpy(Xg))
         assert np.allclose(nb.cpu().numpy(), nb_ref, rtol=TOL_BF16) and np.allclose(Sb.cpu().numpy(), Sb_ref, rtol=TOL_BF16, atol=TOL_BF16 * np.abs(Sb_ref).max() * 0.05)
+        # the same output gradients as those of an embedding table: few ids (long groups), many ids, ids outside the table
+        V = int(rng.choice([2, 17, 5000]))
+        ids = torch.from_numpy(rng.integers(-2, V + 3, size=(B, T)).astype(np.int32)).to(DEV)
+        ne = torch.zeros(B, device=DEV)
+        ctx.embedding_sqnorm(ids, D, V, ne)
+        torch.cuda.synchronize()
+        ne_ref, _ = O.embedding_terms(ids.cpu().numpy(), W.to_numpy(D), V)
+        assert np.allclose(ne.cpu().numpy(), ne_ref, rtol=TOL_BF16, atol=1e-30), f"embedding case {case}: B={B} T={T} d={d_out} V={V}"
     assert ctx.device_status() == 0
